@@ -1,0 +1,146 @@
+/*
+ * pop.h - C ABI of the POP (partition-guided online pruning) hot path for one
+ * SwiGLU FFN / MoE expert block on an NVIDIA B200 (sm_100a).
+ *
+ * The paper states the method in two stages (Sec. 3.3, Sec. 3.4):
+ *   prefill : score every intermediate channel from the whole prompt (Eq. 3) and split the
+ *             channels into Retained / Candidate / Pruned regions around the pruning
+ *             threshold;
+ *   decode  : per step, run the block's first projections over Retained + Candidate only,
+ *             score the Candidate channels from this step's activations, switch on the k
+ *             best of them, and finish the block over Retained + selected channels.
+ * The paper defines no API; the two main calls below follow that statement of the problem.
+ *
+ * Conventions
+ *   d  hidden size, N intermediate size (the N prunable channels), L prompt tokens with the
+ *   batch folded in, B decode batch.  Wg, Wu are [N, d] row-major (row i = channel i); Wd is
+ *   [d, N] row-major (column i = channel i).  f(x) = silu(Wg x) * (Wu x).
+ *   All data pointers are DEVICE pointers unless a parameter is named h_* (host).
+ *   Every function returns an int status (POP_OK == 0, errors negative).  Nothing throws,
+ *   aborts or synchronises the device unless stated; device work is enqueued on the
+ *   cudaStream_t passed as `cuda_stream` (NULL = the legacy default stream).
+ *   A partition is used by one stream at a time.
+ */
+#ifndef POP_H_
+#define POP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define POP_OK                 0
+#define POP_ERR_INVALID_ARG   -1   /* null pointer, size out of range, ratios invalid, k > n_cand ... */
+#define POP_ERR_UNSUPPORTED   -2   /* dtype / shape / batch outside what the kernels handle          */
+#define POP_ERR_ALLOC         -3   /* device or host allocation failed                                */
+#define POP_ERR_CUDA          -4   /* a CUDA runtime call failed; see pop_last_cuda_error()           */
+#define POP_ERR_TIMEOUT       -5   /* a bounded device-side wait expired (reported by pop_partition_check) */
+
+#define POP_MAX_BATCH          8   /* largest decode batch B a partition's scratch is sized for       */
+
+typedef enum { POP_F32 = 0, POP_BF16 = 1 } pop_dtype_t;
+
+/* Fractions of the N channels put into each region; each >= 0, candidate + pruned <= 1. */
+typedef struct { double retained, candidate, pruned; } pop_ratios_t;
+
+/* Opaque, library-owned: repacked weights, region indices, prefill scores, decode scratch. */
+typedef struct pop_partition pop_partition_t;
+
+/* ---- library information (host only) ------------------------------------------------------- */
+const char* pop_version(void);
+const char* pop_status_string(int status);
+/* Text of the last CUDA runtime error seen by this thread inside the library ("" if none). */
+const char* pop_last_cuda_error(void);
+
+/*
+ * Region sizes for N channels (Sec. 3.3: thresholds at the (r - delta) and (r + delta) quantiles;
+ * taken by rank so that the sizes are exact):
+ *   n_pruned = floor(pruned * N + 1e-9), n_cand = floor(candidate * N + 1e-9),
+ *   n_ret = N - n_cand - n_pruned, k_default = floor(n_cand / 2).
+ * Host only. Any output pointer may be NULL.  POP_ERR_INVALID_ARG on bad ratios or N <= 0.
+ */
+int pop_region_sizes(int N, pop_ratios_t ratios, int* n_ret, int* n_cand, int* n_pruned, int* k_default);
+
+/*
+ * Prefilling stage (Sec. 3.3 "Prefilling Stage"; score = Eq. 3 of Sec. 3.4).
+ *   X [L, d], Wg [N, d], Wu [N, d], Wd [d, N]: row-major device arrays of `dtype`, read-only,
+ *   owned by the caller; they may be freed once the stream has passed this call (the
+ *   partition keeps its own repacked copy of the live rows).
+ * Computes, on `cuda_stream`:
+ *   H[t, i] = silu(Wg[i].X[t]) * (Wu[i].X[t]);  s_i = sqrt(sum_t H[t,i]^2);
+ *   I_i = s_i * ||Wd[:, i]||_2   (Eq. 3 with W = the down projection, whose input channel i
+ *   is intermediate channel i);
+ *   ranks channels by (I_i descending, i ascending): the first n_ret are Retained, the next
+ *   n_cand Candidate, the rest Pruned (sizes as pop_region_sizes);
+ *   repacks Wg/Wu rows and Wd columns of Retained then Candidate channels contiguously.
+ * The ranking is decided on fp64 scores.  *out receives a new partition (destroy it with
+ * pop_partition_destroy).  Allocates device memory (about (n_ret + n_cand) * 3 * d elements).
+ * Requirements: d * sizeof(element) a multiple of 16; pointers 16-byte aligned; L >= 1.
+ * Errors: POP_ERR_INVALID_ARG, POP_ERR_UNSUPPORTED, POP_ERR_ALLOC, POP_ERR_CUDA.
+ */
+int pop_prefill_partition(const void* X, int L, int d,
+                          const void* Wg, const void* Wu, const void* Wd, int N,
+                          pop_dtype_t dtype, pop_ratios_t ratios,
+                          void* cuda_stream, pop_partition_t** out);
+
+/*
+ * Build a partition from caller-chosen regions instead of prefill scores (the regions of
+ * Sec. 3.3 given explicitly).  h_ret [n_ret] and h_cand [n_cand] are HOST arrays of channel
+ * ids, each strictly ascending, disjoint, in [0, N); channels in neither are Pruned.
+ * The prefill scores of such a partition are all zero.  Same requirements and errors as above.
+ */
+int pop_partition_from_indices(const void* Wg, const void* Wu, const void* Wd, int N, int d,
+                               pop_dtype_t dtype,
+                               const int32_t* h_ret, int n_ret, const int32_t* h_cand, int n_cand,
+                               void* cuda_stream, pop_partition_t** out);
+
+/* Sizes of the three regions (host values, available as soon as the partition exists). */
+int pop_partition_sizes(const pop_partition_t* p, int* n_ret, int* n_cand, int* n_pruned);
+
+/*
+ * Region index arrays: DEVICE int32 arrays owned by the partition, each ascending by channel
+ * id, of the sizes above (Sec. 3.3: R, C, P are disjoint and cover all channels).  Valid on the
+ * stream the partition was built on (or after synchronising it).  Any output may be NULL.
+ */
+int pop_partition_indices(const pop_partition_t* p, const int32_t** d_ret,
+                          const int32_t** d_cand, const int32_t** d_pruned);
+
+/* Prefill importance scores I_i (Eq. 3), DEVICE double [N], owned by the partition. */
+int pop_partition_scores(const pop_partition_t* p, const double** d_scores);
+
+/* Shape of a partition: any output may be NULL. */
+int pop_partition_shape(const pop_partition_t* p, int* d, int* N, pop_dtype_t* dtype);
+
+/*
+ * Synchronises the partition's device (cudaDeviceSynchronize) and reports whether any decode
+ * step on it gave up a bounded wait since the last check: POP_OK or POP_ERR_TIMEOUT.  After a
+ * timeout the outputs of that step are undefined; the partition stays usable.
+ */
+int pop_partition_check(pop_partition_t* p);
+
+/* Frees everything the partition owns.  The caller must have synchronised its stream. */
+int pop_partition_destroy(pop_partition_t* p);
+
+/*
+ * One decoding step (Sec. 3.3 "Decoding Stage"; Sec. 3.4: forward over R u C, scores of the
+ * candidates from H_t, selection, final computation over R u selected only).
+ *   x [B, d] -> y [B, d], device arrays of the partition's dtype, caller-owned; 1 <= B <= POP_MAX_BATCH.
+ *   h[b, i] = silu(Wg[i].x[b]) * (Wu[i].x[b]) for i in R u C;
+ *   score_i = ||Wd[:, i]||_2 * sqrt(sum_b h[b, i]^2) for i in C (one mask shared by the batch);
+ *   M = the k_candidate candidates with the largest (score descending, channel id ascending),
+ *       decided on fp64 scores;
+ *   y[b] = sum over i in R u M of Wd[:, i] * h[b, i]   (fp32 accumulation).
+ *   mask_out: uint8 [n_cand], 1 where the candidate in that slot (slot order = the d_cand array)
+ *             was selected; may be NULL.
+ *   sel_out : int32 [k_candidate], channel ids of the selected candidates, ascending; may be NULL.
+ * No allocation, no host synchronisation.  0 <= k_candidate <= n_cand.
+ * Errors: POP_ERR_INVALID_ARG, POP_ERR_UNSUPPORTED (B too large for the shape), POP_ERR_CUDA.
+ */
+int pop_decode_step(pop_partition_t* p, const void* x, int B, int k_candidate,
+                    void* y, uint8_t* mask_out, int32_t* sel_out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POP_H_ */

@@ -1,0 +1,267 @@
+// C ABI of the POP library: argument checking, partition life cycle, stage sequencing.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "pop_common.cuh"
+
+static thread_local char g_cuda_err[256] = "";
+
+void pop_set_cuda_error(cudaError_t e, const char* what) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+    (void)cudaGetLastError();   // clear the sticky-free error state
+}
+
+extern "C" const char* pop_version(void) { return "pop-b200 0.1.0 (sm_100a)"; }
+
+extern "C" const char* pop_last_cuda_error(void) { return g_cuda_err; }
+
+extern "C" const char* pop_status_string(int s) {
+    switch (s) {
+        case POP_OK: return "POP_OK";
+        case POP_ERR_INVALID_ARG: return "POP_ERR_INVALID_ARG";
+        case POP_ERR_UNSUPPORTED: return "POP_ERR_UNSUPPORTED";
+        case POP_ERR_ALLOC: return "POP_ERR_ALLOC";
+        case POP_ERR_CUDA: return "POP_ERR_CUDA";
+        case POP_ERR_TIMEOUT: return "POP_ERR_TIMEOUT";
+        default: return "POP_ERR_UNKNOWN";
+    }
+}
+
+extern "C" int pop_region_sizes(int N, pop_ratios_t r, int* n_ret, int* n_cand, int* n_pruned, int* k_default) {
+    if (N <= 0) return POP_ERR_INVALID_ARG;
+    if (!(r.retained >= 0.0) || !(r.candidate >= 0.0) || !(r.pruned >= 0.0)) return POP_ERR_INVALID_ARG;
+    if (r.retained + r.candidate + r.pruned > 1.0 + 1e-9 || r.candidate + r.pruned > 1.0 + 1e-9)
+        return POP_ERR_INVALID_ARG;
+    const int np = (int)floor(r.pruned * (double)N + 1e-9);
+    const int nc = (int)floor(r.candidate * (double)N + 1e-9);
+    const int nr = N - np - nc;
+    if (nr < 0) return POP_ERR_INVALID_ARG;
+    if (n_ret) *n_ret = nr;
+    if (n_cand) *n_cand = nc;
+    if (n_pruned) *n_pruned = np;
+    if (k_default) *k_default = nc / 2;
+    return POP_OK;
+}
+
+static bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
+
+static int check_shape(int d, int N, pop_dtype_t dt) {
+    if (d <= 0 || N <= 0) return POP_ERR_INVALID_ARG;
+    if (dt != POP_F32 && dt != POP_BF16) return POP_ERR_UNSUPPORTED;
+    const int es = dt == POP_F32 ? 4 : 2;
+    if (((size_t)d * es) % 16 != 0) return POP_ERR_UNSUPPORTED;
+    if ((size_t)d * es > 65536) return POP_ERR_UNSUPPORTED;
+    return POP_OK;
+}
+
+template <typename P>
+static int dev_alloc(P** ptr, size_t bytes) {
+    *ptr = nullptr;
+    if (bytes == 0) bytes = 16;
+    POP_CUDA(cudaMalloc((void**)ptr, bytes));
+    return POP_OK;
+}
+
+static void partition_free(pop_partition* p) {
+    if (!p) return;
+    cudaFree(p->GU); cudaFree(p->WdT); cudaFree(p->idx_ret); cudaFree(p->idx_cand); cudaFree(p->idx_pruned);
+    cudaFree(p->scores); cudaFree(p->norm_cand); cudaFree(p->h); cudaFree(p->keys); cudaFree(p->y_acc);
+    cudaFree(p->sel_slots); cudaFree(p->sync);
+    free(p);
+}
+
+// Allocates the partition's buffers for given region sizes (contents undefined except zeroed scratch).
+static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, cudaStream_t st, pop_partition** out) {
+    pop_partition* p = (pop_partition*)calloc(1, sizeof(pop_partition));
+    if (!p) return POP_ERR_ALLOC;
+    int rc = POP_OK;
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaGetDevice"); free(p); return POP_ERR_CUDA; }
+    p->d = d; p->N = N; p->dtype = dt; p->es = dt == POP_F32 ? 4 : 2;
+    p->n_ret = n_ret; p->n_cand = n_cand; p->n_pruned = N - n_ret - n_cand; p->n_rc = n_ret + n_cand;
+    cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+    cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device);
+    cudaDeviceGetAttribute(&p->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
+    const size_t row = (size_t)d * p->es;
+#define TRY(x) do { rc = (x); if (rc != POP_OK) { partition_free(p); return rc; } } while (0)
+    TRY(dev_alloc(&p->GU, (size_t)p->n_rc * 2 * row));
+    TRY(dev_alloc(&p->WdT, (size_t)p->n_rc * row));
+    TRY(dev_alloc(&p->idx_ret, sizeof(int32_t) * (size_t)n_ret));
+    TRY(dev_alloc(&p->idx_cand, sizeof(int32_t) * (size_t)n_cand));
+    TRY(dev_alloc(&p->idx_pruned, sizeof(int32_t) * (size_t)p->n_pruned));
+    TRY(dev_alloc(&p->scores, sizeof(double) * (size_t)N));
+    TRY(dev_alloc(&p->norm_cand, sizeof(double) * (size_t)n_cand));
+    TRY(dev_alloc(&p->h, sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->n_rc > 0 ? p->n_rc : 1)));
+    TRY(dev_alloc(&p->keys, sizeof(u64) * (size_t)n_cand));
+    TRY(dev_alloc(&p->y_acc, sizeof(float) * (size_t)POP_MAX_BATCH * d));
+    TRY(dev_alloc(&p->sel_slots, sizeof(int32_t) * (size_t)n_cand));
+    TRY(dev_alloc(&p->sync, sizeof(u32) * SYNC_WORDS));
+#undef TRY
+    e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->scores, 0, sizeof(double) * (size_t)N, st);
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free(p); return POP_ERR_CUDA; }
+    *out = p;
+    return POP_OK;
+}
+
+extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg, const void* Wu, const void* Wd,
+                                     int N, pop_dtype_t dtype, pop_ratios_t ratios, void* cuda_stream,
+                                     pop_partition_t** out) {
+    if (!out) return POP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!X || !Wg || !Wu || !Wd || L <= 0) return POP_ERR_INVALID_ARG;
+    int rc = check_shape(d, N, dtype);
+    if (rc != POP_OK) return rc;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd)) return POP_ERR_INVALID_ARG;
+    int n_ret, n_cand, n_pruned;
+    rc = pop_region_sizes(N, ratios, &n_ret, &n_cand, &n_pruned, nullptr);
+    if (rc != POP_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+
+    pop_partition* p = nullptr;
+    rc = partition_alloc(d, N, dtype, n_ret, n_cand, st, &p);
+    if (rc != POP_OK) return rc;
+
+    // temporaries: column norms and activation energies, freed in stream order
+    double *norm = nullptr, *s2 = nullptr;
+    cudaError_t e = cudaMallocAsync((void**)&norm, sizeof(double) * (size_t)N, st);
+    if (e == cudaSuccess) e = cudaMallocAsync((void**)&s2, sizeof(double) * (size_t)N, st);
+    if (e != cudaSuccess) {
+        pop_set_cuda_error(e, "cudaMallocAsync");
+        if (norm) cudaFreeAsync(norm, st);
+        partition_free(p);
+        return POP_ERR_ALLOC;
+    }
+    rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
+    if (rc == POP_OK) rc = pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
+    if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, p->scores, st);
+    if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->idx_ret, p->idx_cand, p->idx_pruned, st);
+    if (rc == POP_OK) rc = pop_launch_repack(p, Wg, Wu, Wd, norm, st);
+    cudaFreeAsync(norm, st);
+    cudaFreeAsync(s2, st);
+    if (rc != POP_OK) { cudaStreamSynchronize(st); partition_free(p); return rc; }
+    *out = p;
+    return POP_OK;
+}
+
+extern "C" int pop_partition_from_indices(const void* Wg, const void* Wu, const void* Wd, int N, int d,
+                                          pop_dtype_t dtype, const int32_t* h_ret, int n_ret,
+                                          const int32_t* h_cand, int n_cand, void* cuda_stream,
+                                          pop_partition_t** out) {
+    if (!out) return POP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!Wg || !Wu || !Wd || n_ret < 0 || n_cand < 0) return POP_ERR_INVALID_ARG;
+    if ((n_ret > 0 && !h_ret) || (n_cand > 0 && !h_cand)) return POP_ERR_INVALID_ARG;
+    int rc = check_shape(d, N, dtype);
+    if (rc != POP_OK) return rc;
+    if (!aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd)) return POP_ERR_INVALID_ARG;
+    if ((long long)n_ret + n_cand > N) return POP_ERR_INVALID_ARG;
+    // ascending, in range, disjoint
+    unsigned char* seen = (unsigned char*)calloc((size_t)N, 1);
+    if (!seen) return POP_ERR_ALLOC;
+    bool ok = true;
+    for (int pass = 0; pass < 2 && ok; ++pass) {
+        const int32_t* a = pass ? h_cand : h_ret;
+        const int n = pass ? n_cand : n_ret;
+        for (int i = 0; i < n; ++i) {
+            if (a[i] < 0 || a[i] >= N || (i > 0 && a[i] <= a[i - 1]) || seen[a[i]]) { ok = false; break; }
+            seen[a[i]] = 1;
+        }
+    }
+    int32_t* h_pruned = nullptr;
+    const int n_pruned = N - n_ret - n_cand;
+    if (ok) {
+        h_pruned = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n_pruned > 0 ? n_pruned : 1));
+        if (h_pruned) { int q = 0; for (int i = 0; i < N; ++i) if (!seen[i]) h_pruned[q++] = i; }
+    }
+    free(seen);
+    if (!ok) return POP_ERR_INVALID_ARG;
+    if (!h_pruned) return POP_ERR_ALLOC;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    pop_partition* p = nullptr;
+    rc = partition_alloc(d, N, dtype, n_ret, n_cand, st, &p);
+    if (rc != POP_OK) { free(h_pruned); return rc; }
+    cudaError_t e = cudaSuccess;
+    if (n_ret) e = cudaMemcpyAsync(p->idx_ret, h_ret, sizeof(int32_t) * (size_t)n_ret, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && n_cand) e = cudaMemcpyAsync(p->idx_cand, h_cand, sizeof(int32_t) * (size_t)n_cand, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && n_pruned) e = cudaMemcpyAsync(p->idx_pruned, h_pruned, sizeof(int32_t) * (size_t)n_pruned, cudaMemcpyHostToDevice, st);
+    // the host arrays are pageable: wait so that the caller (and h_pruned) may go away
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    free(h_pruned);
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "index upload"); partition_free(p); return POP_ERR_CUDA; }
+    double* norm = nullptr;
+    e = cudaMallocAsync((void**)&norm, sizeof(double) * (size_t)N, st);
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMallocAsync"); partition_free(p); return POP_ERR_ALLOC; }
+    rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
+    if (rc == POP_OK) rc = pop_launch_repack(p, Wg, Wu, Wd, norm, st);
+    cudaFreeAsync(norm, st);
+    if (rc != POP_OK) { cudaStreamSynchronize(st); partition_free(p); return rc; }
+    *out = p;
+    return POP_OK;
+}
+
+extern "C" int pop_partition_sizes(const pop_partition_t* p, int* n_ret, int* n_cand, int* n_pruned) {
+    if (!p) return POP_ERR_INVALID_ARG;
+    if (n_ret) *n_ret = p->n_ret;
+    if (n_cand) *n_cand = p->n_cand;
+    if (n_pruned) *n_pruned = p->n_pruned;
+    return POP_OK;
+}
+
+extern "C" int pop_partition_indices(const pop_partition_t* p, const int32_t** d_ret, const int32_t** d_cand,
+                                     const int32_t** d_pruned) {
+    if (!p) return POP_ERR_INVALID_ARG;
+    if (d_ret) *d_ret = p->idx_ret;
+    if (d_cand) *d_cand = p->idx_cand;
+    if (d_pruned) *d_pruned = p->idx_pruned;
+    return POP_OK;
+}
+
+extern "C" int pop_partition_scores(const pop_partition_t* p, const double** d_scores) {
+    if (!p || !d_scores) return POP_ERR_INVALID_ARG;
+    *d_scores = p->scores;
+    return POP_OK;
+}
+
+extern "C" int pop_partition_shape(const pop_partition_t* p, int* d, int* N, pop_dtype_t* dtype) {
+    if (!p) return POP_ERR_INVALID_ARG;
+    if (d) *d = p->d;
+    if (N) *N = p->N;
+    if (dtype) *dtype = p->dtype;
+    return POP_OK;
+}
+
+extern "C" int pop_partition_check(pop_partition_t* p) {
+    if (!p) return POP_ERR_INVALID_ARG;
+    POP_CUDA(cudaDeviceSynchronize());
+    u32 flag = 0;
+    POP_CUDA(cudaMemcpy(&flag, p->sync + SYNC_ERROR, sizeof(u32), cudaMemcpyDeviceToHost));
+    if (flag) {
+        // leave the partition usable: clear counters and the accumulator
+        POP_CUDA(cudaMemset(p->sync, 0, sizeof(u32) * SYNC_WORDS));
+        POP_CUDA(cudaMemset(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * p->d));
+        return POP_ERR_TIMEOUT;
+    }
+    return POP_OK;
+}
+
+extern "C" int pop_partition_destroy(pop_partition_t* p) {
+    if (!p) return POP_ERR_INVALID_ARG;
+    partition_free(p);
+    return POP_OK;
+}
+
+extern "C" int pop_decode_step(pop_partition_t* p, const void* x, int B, int k_candidate, void* y,
+                               uint8_t* mask_out, int32_t* sel_out, void* cuda_stream) {
+    if (!p || !x || !y) return POP_ERR_INVALID_ARG;
+    if (B < 1 || k_candidate < 0 || k_candidate > p->n_cand) return POP_ERR_INVALID_ARG;
+    if (B > POP_MAX_BATCH) return POP_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(y)) return POP_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int rc = pop_launch_decode(p, x, B, k_candidate, y, mask_out, sel_out, st);
+    if (rc == POP_ERR_UNSUPPORTED) rc = pop_launch_decode_simple(p, x, B, k_candidate, y, mask_out, sel_out, st);
+    return rc;
+}

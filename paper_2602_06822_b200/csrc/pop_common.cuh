@@ -1,0 +1,118 @@
+// Shared declarations of the POP CUDA library (internal; the public C ABI is include/pop.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "pop.h"
+
+typedef unsigned long long u64;
+typedef unsigned int u32;
+
+// ---------------------------------------------------------------------------------------------
+// Partition object (host struct; every pointer below is device memory owned by it).
+//
+// Repacked layout ("slots"): slot s in [0, n_ret) is Retained channel idx_ret[s]; slot
+// n_ret + c is Candidate channel idx_cand[c].  n_rc = n_ret + n_cand.
+//   GU  [n_rc][2][d]  gate row then up row of the slot's channel, contiguous (one 2*d*es block)
+//   WdT [n_rc][d]     column of the down projection of the slot's channel, as a contiguous row
+// ---------------------------------------------------------------------------------------------
+struct pop_partition {
+    int device;
+    int d, N;
+    pop_dtype_t dtype;
+    int es;                       // element size in bytes
+    int n_ret, n_cand, n_pruned, n_rc;
+
+    void* GU;
+    void* WdT;
+    int32_t* idx_ret;
+    int32_t* idx_cand;
+    int32_t* idx_pruned;
+    double* scores;               // [N] prefill I_i
+    double* norm_cand;            // [n_cand] ||Wd[:, i]||_2 of the candidate channels
+
+    // decode scratch (no allocation at decode time)
+    float* h;                     // [POP_MAX_BATCH][n_rc] intermediate activations of this step
+    u64* keys;                    // [n_cand] candidate scores as ordered 64-bit keys
+    float* y_acc;                 // [POP_MAX_BATCH][d] fp32 accumulator, zero between steps
+    int32_t* sel_slots;           // [n_cand] selected candidate slots (ascending), this step
+    u32* sync;                    // [16] counters / flags, see pop_decode.cu
+    int sm_count;
+    int coop;                     // device supports cooperative launch
+    int max_smem_optin;
+};
+
+// sync[] word assignment
+enum { SYNC_BARRIER = 0, SYNC_TICKET = 1, SYNC_ERROR = 2, SYNC_WORK = 3, SYNC_WORDS = 16 };
+
+// ---------------------------------------------------------------------------------------------
+// error plumbing
+// ---------------------------------------------------------------------------------------------
+void pop_set_cuda_error(cudaError_t e, const char* what);
+
+#define POP_CUDA(call)                                                    \
+    do {                                                                  \
+        cudaError_t e__ = (call);                                         \
+        if (e__ != cudaSuccess) {                                         \
+            pop_set_cuda_error(e__, #call);                               \
+            return (e__ == cudaErrorMemoryAllocation) ? POP_ERR_ALLOC : POP_ERR_CUDA; \
+        }                                                                 \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// launchers implemented in the .cu files (host functions; all enqueue on `st`)
+// ---------------------------------------------------------------------------------------------
+// pop_prefill.cu
+int pop_launch_colnorm(const void* Wd, int d, int N, pop_dtype_t dt, double* norm /*[N]*/, cudaStream_t st);
+int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, const void* Wu, int N,
+                                pop_dtype_t dt, const int32_t* chan_list /*NULL = all*/, int n_list,
+                                double* s2 /*[N], entries of listed channels are overwritten*/, cudaStream_t st);
+int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st);
+int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand,
+                         int32_t* idx_ret, int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);
+int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
+                      const double* norm /*[N]*/, cudaStream_t st);
+// pop_decode_simple.cu (multi-kernel path, any accepted shape)
+int pop_launch_decode_simple(pop_partition* p, const void* x, int B, int k, void* y,
+                             uint8_t* mask_out, int32_t* sel_out, cudaStream_t st);
+// pop_decode.cu (fused persistent kernel; returns POP_ERR_UNSUPPORTED for shapes it does not take)
+int pop_launch_decode(pop_partition* p, const void* x, int B, int k, void* y,
+                      uint8_t* mask_out, int32_t* sel_out, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int VEC = 4;                       // elements per 16-byte vector
+    __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[4]) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ float to_f32(float v) { return v; }
+    __device__ static __forceinline__ float from_f32(float v) { return v; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int VEC = 8;
+    __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+    __device__ static __forceinline__ __nv_bfloat16 from_f32(float v) { return __float2bfloat16_rn(v); }
+};
+
+// silu(z) = z / (1 + exp(-z)), in the precision of the argument.
+__device__ __forceinline__ double silu_f64(double z) { return z / (1.0 + exp(-z)); }
+__device__ __forceinline__ float silu_f32(float z) { return z / (1.0f + expf(-z)); }
+
+// Scores are non-negative finite doubles: their bit patterns order like the values.
+__device__ __forceinline__ u64 score_key(double s) { return (u64)__double_as_longlong(s); }
+
+#endif  // __CUDACC__

@@ -1,0 +1,277 @@
+// Prefilling stage of POP (Sec. 3.3 "Prefilling Stage"; score of Sec. 3.4 Eq. 3):
+//   column norms of the down projection, per-channel activation energy over the prompt,
+//   importance scores, rank-select into Retained / Candidate / Pruned, weight repack.
+#include "pop_common.cuh"
+#include "pop_select.cuh"
+
+// ---------------------------------------------------------------------------------------------
+// n_i = ||Wd[:, i]||_2  (the weight factor of Eq. 3: ||W[:, i] * s_i||_2 = |s_i| * ||W[:, i]||_2).
+// Block (32 columns x 32 row strips); every column is summed in the same fixed order, so equal
+// columns give bit-equal norms.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(1024) colnorm_kernel(const T* __restrict__ Wd, int d, int N,
+                                                       double* __restrict__ norm) {
+    __shared__ double part[32][33];
+    const int cx = threadIdx.x, ry = threadIdx.y;
+    const int c = blockIdx.x * 32 + cx;
+    double acc = 0.0;
+    if (c < N) {
+        for (int j = ry; j < d; j += 32) {
+            double v = (double)Elem<T>::to_f32(Wd[(size_t)j * N + c]);
+            acc = fma(v, v, acc);
+        }
+    }
+    part[ry][cx] = acc;
+    __syncthreads();
+    if (ry == 0 && c < N) {
+        double s = 0.0;
+#pragma unroll 1
+        for (int r = 0; r < 32; ++r) s += part[r][cx];
+        norm[c] = sqrt(s);
+    }
+}
+
+int pop_launch_colnorm(const void* Wd, int d, int N, pop_dtype_t dt, double* norm, cudaStream_t st) {
+    dim3 blk(32, 32), grd((N + 31) / 32);
+    if (dt == POP_F32) colnorm_kernel<float><<<grd, blk, 0, st>>>((const float*)Wd, d, N, norm);
+    else colnorm_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, d, N, norm);
+    POP_CUDA(cudaGetLastError());
+    return POP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exact (fp64) activation energy  s2[i] = sum_t H[t, i]^2,  H[t, i] = silu(Wg[i].X[t]) * (Wu[i].X[t])
+// for the channels in chan_list (all channels when chan_list == NULL).
+//
+// One block owns 32 channels and walks over all tokens in tiles of 32; K is consumed in chunks
+// of 32 staged in shared memory as doubles.  Thread (tx, ty) of the 16 x 16 block computes
+// channels {tx, tx+16} x tokens {ty, ty+16}.  The per-channel sum over tokens is taken in a
+// fixed order that is the same for every channel.
+// ---------------------------------------------------------------------------------------------
+#define S2_CT 32
+#define S2_TT 32
+#define S2_KT 32
+
+template <typename T>
+__global__ void __launch_bounds__(256) prefill_s2_exact_kernel(
+    const T* __restrict__ X, int L, int d, const T* __restrict__ Wg, const T* __restrict__ Wu, int N,
+    const int32_t* __restrict__ chan_list, int n_list, double* __restrict__ s2) {
+    __shared__ double Xs[S2_TT][S2_KT + 1];
+    __shared__ double Gs[S2_CT][S2_KT + 1];
+    __shared__ double Us[S2_CT][S2_KT + 1];
+    __shared__ int chan[S2_CT];
+    __shared__ double red[16][S2_CT + 1];
+
+    const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+    const int c0 = blockIdx.x * S2_CT;
+    if (tid < S2_CT) {
+        int li = c0 + tid;
+        chan[tid] = (li < n_list) ? (chan_list ? chan_list[li] : li) : -1;
+    }
+    __syncthreads();
+
+    double e[2] = {0.0, 0.0};                     // energy of channels tx, tx+16 over this thread's tokens
+    for (int t0 = 0; t0 < L; t0 += S2_TT) {
+        double g[2][2] = {{0, 0}, {0, 0}}, u[2][2] = {{0, 0}, {0, 0}};
+        for (int k0 = 0; k0 < d; k0 += S2_KT) {
+            // stage X[t0..+32][k0..+32], Wg/Wu[chan][k0..+32] as doubles (zero outside bounds)
+            for (int idx = tid; idx < S2_TT * S2_KT; idx += 256) {
+                int r = idx / S2_KT, kk = idx % S2_KT, k = k0 + kk;
+                int t = t0 + r;
+                Xs[r][kk] = (t < L && k < d) ? (double)Elem<T>::to_f32(X[(size_t)t * d + k]) : 0.0;
+                int ch = chan[r];
+                bool ok = ch >= 0 && k < d;
+                Gs[r][kk] = ok ? (double)Elem<T>::to_f32(Wg[(size_t)ch * d + k]) : 0.0;
+                Us[r][kk] = ok ? (double)Elem<T>::to_f32(Wu[(size_t)ch * d + k]) : 0.0;
+            }
+            __syncthreads();
+#pragma unroll 8
+            for (int kk = 0; kk < S2_KT; ++kk) {
+                double x0 = Xs[ty][kk], x1 = Xs[ty + 16][kk];
+                double g0 = Gs[tx][kk], g1 = Gs[tx + 16][kk];
+                double u0 = Us[tx][kk], u1 = Us[tx + 16][kk];
+                g[0][0] = fma(g0, x0, g[0][0]); g[0][1] = fma(g0, x1, g[0][1]);
+                g[1][0] = fma(g1, x0, g[1][0]); g[1][1] = fma(g1, x1, g[1][1]);
+                u[0][0] = fma(u0, x0, u[0][0]); u[0][1] = fma(u0, x1, u[0][1]);
+                u[1][0] = fma(u1, x0, u[1][0]); u[1][1] = fma(u1, x1, u[1][1]);
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                // tokens beyond L contribute silu(0) * 0 = 0
+                double h = silu_f64(g[c][t]) * u[c][t];
+                e[c] = fma(h, h, e[c]);
+            }
+    }
+    red[ty][tx] = e[0];
+    red[ty][tx + 16] = e[1];
+    __syncthreads();
+    if (tid < S2_CT && chan[tid] >= 0) {
+        double s = 0.0;
+#pragma unroll 1
+        for (int r = 0; r < 16; ++r) s += red[r][tid];
+        s2[chan[tid]] = s;
+    }
+}
+
+int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, const void* Wu, int N,
+                                pop_dtype_t dt, const int32_t* chan_list, int n_list, double* s2,
+                                cudaStream_t st) {
+    if (n_list <= 0) return POP_OK;
+    dim3 grd((n_list + S2_CT - 1) / S2_CT);
+    if (dt == POP_F32)
+        prefill_s2_exact_kernel<float><<<grd, 256, 0, st>>>((const float*)X, L, d, (const float*)Wg,
+                                                            (const float*)Wu, N, chan_list, n_list, s2);
+    else
+        prefill_s2_exact_kernel<__nv_bfloat16><<<grd, 256, 0, st>>>(
+            (const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, N,
+            chan_list, n_list, s2);
+    POP_CUDA(cudaGetLastError());
+    return POP_OK;
+}
+
+// I_i = sqrt(s2_i) * n_i   (Eq. 3)
+__global__ void scores_kernel(const double* __restrict__ s2, const double* __restrict__ norm, int N,
+                              double* __restrict__ scores) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < N) scores[i] = sqrt(s2[i]) * norm[i];
+}
+
+int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st) {
+    scores_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2, norm, N, scores);
+    POP_CUDA(cudaGetLastError());
+    return POP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Partition (Sec. 3.3): rank by (score descending, channel id ascending); the first n_ret
+// channels are Retained, the next n_cand Candidate, the rest Pruned.  One block: two radix
+// selects give the two rank boundaries (the tau_high and tau_low thresholds of the paper, with
+// ties split by channel id), then one ordered walk writes the three ascending index lists.
+// ---------------------------------------------------------------------------------------------
+#define PART_NT 1024
+
+__global__ void __launch_bounds__(PART_NT) partition_kernel(const double* __restrict__ scores, int N,
+                                                            int n_ret, int n_cand,
+                                                            int32_t* __restrict__ idx_ret,
+                                                            int32_t* __restrict__ idx_cand,
+                                                            int32_t* __restrict__ idx_pruned) {
+    __shared__ u32 sm[POP_SELECT_SMEM_WORDS(PART_NT)];
+    const int tid = threadIdx.x;
+    const u64* keys = reinterpret_cast<const u64*>(scores);   // non-negative doubles order like their bits
+
+    u64 thr1 = ~0ull, thr2 = ~0ull;
+    int ne1 = 0, ne2 = 0;
+    if (n_ret > 0) radix_select_kth<PART_NT>(keys, N, n_ret, sm, tid, 0, thr1, ne1);
+    if (n_ret + n_cand > 0) radix_select_kth<PART_NT>(keys, N, n_ret + n_cand, sm, tid, 0, thr2, ne2);
+
+    const int per = (N + PART_NT - 1) / PART_NT;
+    const int lo = min(N, tid * per), hi = min(N, lo + per);
+    int eq1 = 0, eq2 = 0;
+    for (int i = lo; i < hi; ++i) { u64 k = keys[i]; eq1 += (k == thr1); eq2 += (k == thr2); }
+    int tot;
+    const int eb1 = group_excl_scan<PART_NT>(eq1, sm, tid, 0, tot);
+    const int eb2 = group_excl_scan<PART_NT>(eq2, sm, tid, 0, tot);
+    int cR = 0, cC = 0, cP = 0, e1 = eb1, e2 = eb2;
+    for (int i = lo; i < hi; ++i) {
+        u64 k = keys[i];
+        bool top1 = k > thr1, top2 = k > thr2;
+        if (k == thr1) { top1 = e1 < ne1; ++e1; }
+        if (k == thr2) { top2 = e2 < ne2; ++e2; }
+        if (top1) ++cR; else if (top2) ++cC; else ++cP;
+    }
+    int pR = group_excl_scan<PART_NT>(cR, sm, tid, 0, tot);
+    int pC = group_excl_scan<PART_NT>(cC, sm, tid, 0, tot);
+    int pP = group_excl_scan<PART_NT>(cP, sm, tid, 0, tot);
+    e1 = eb1; e2 = eb2;
+    for (int i = lo; i < hi; ++i) {
+        u64 k = keys[i];
+        bool top1 = k > thr1, top2 = k > thr2;
+        if (k == thr1) { top1 = e1 < ne1; ++e1; }
+        if (k == thr2) { top2 = e2 < ne2; ++e2; }
+        if (top1) idx_ret[pR++] = i; else if (top2) idx_cand[pC++] = i; else idx_pruned[pP++] = i;
+    }
+}
+
+int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* idx_ret,
+                         int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st) {
+    partition_kernel<<<1, PART_NT, 0, st>>>(scores, N, n_ret, n_cand, idx_ret, idx_cand, idx_pruned);
+    POP_CUDA(cudaGetLastError());
+    return POP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Repack: live rows of Wg/Wu interleaved per slot, live columns of Wd transposed into rows.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int slot_channel(int s, int n_ret, const int32_t* idx_ret, const int32_t* idx_cand) {
+    return s < n_ret ? idx_ret[s] : idx_cand[s - n_ret];
+}
+
+// one block per slot; rows are d*es bytes, a multiple of 16
+__global__ void __launch_bounds__(256) repack_gu_kernel(const uint4* __restrict__ Wg, const uint4* __restrict__ Wu,
+                                                        int row_vecs, int n_ret,
+                                                        const int32_t* __restrict__ idx_ret,
+                                                        const int32_t* __restrict__ idx_cand,
+                                                        uint4* __restrict__ GU) {
+    const int s = blockIdx.x;
+    const int ch = slot_channel(s, n_ret, idx_ret, idx_cand);
+    const uint4* g = Wg + (size_t)ch * row_vecs;
+    const uint4* u = Wu + (size_t)ch * row_vecs;
+    uint4* o = GU + (size_t)s * 2 * row_vecs;
+    for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
+        o[v] = g[v];
+        o[row_vecs + v] = u[v];
+    }
+}
+
+// WdT[s][j] = Wd[j][channel(s)]: tile of 32 slots x 32 rows through shared memory
+template <typename T>
+__global__ void __launch_bounds__(1024) repack_wdt_kernel(const T* __restrict__ Wd, int d, int N, int n_rc,
+                                                          int n_ret, const int32_t* __restrict__ idx_ret,
+                                                          const int32_t* __restrict__ idx_cand,
+                                                          T* __restrict__ WdT) {
+    __shared__ T tile[32][33];
+    const int s0 = blockIdx.x * 32, j0 = blockIdx.y * 32;
+    int s = s0 + threadIdx.x, j = j0 + threadIdx.y;
+    if (s < n_rc && j < d) {
+        int ch = slot_channel(s, n_ret, idx_ret, idx_cand);
+        tile[threadIdx.y][threadIdx.x] = Wd[(size_t)j * N + ch];
+    }
+    __syncthreads();
+    s = s0 + threadIdx.y; j = j0 + threadIdx.x;
+    if (s < n_rc && j < d) WdT[(size_t)s * d + j] = tile[threadIdx.x][threadIdx.y];
+}
+
+__global__ void gather_norm_kernel(const double* __restrict__ norm, const int32_t* __restrict__ idx_cand,
+                                   int n_cand, double* __restrict__ norm_cand) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < n_cand) norm_cand[c] = norm[idx_cand[c]];
+}
+
+int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
+                      const double* norm, cudaStream_t st) {
+    if (p->n_rc > 0) {
+        const int row_vecs = p->d * p->es / 16;
+        repack_gu_kernel<<<p->n_rc, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, p->n_ret,
+                                                  p->idx_ret, p->idx_cand, (uint4*)p->GU);
+        POP_CUDA(cudaGetLastError());
+        dim3 blk(32, 32), grd((p->n_rc + 31) / 32, (p->d + 31) / 32);
+        if (p->dtype == POP_F32)
+            repack_wdt_kernel<float><<<grd, blk, 0, st>>>((const float*)Wd, p->d, p->N, p->n_rc, p->n_ret,
+                                                          p->idx_ret, p->idx_cand, (float*)p->WdT);
+        else
+            repack_wdt_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_rc,
+                                                                   p->n_ret, p->idx_ret, p->idx_cand,
+                                                                   (__nv_bfloat16*)p->WdT);
+        POP_CUDA(cudaGetLastError());
+    }
+    if (p->n_cand > 0) {
+        gather_norm_kernel<<<(p->n_cand + 255) / 256, 256, 0, st>>>(norm, p->idx_cand, p->n_cand, p->norm_cand);
+        POP_CUDA(cudaGetLastError());
+    }
+    return POP_OK;
+}

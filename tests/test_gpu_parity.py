@@ -1,0 +1,217 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Regions / masks / selected ids bit-exact (near-tie swaps per tests/parity.py),
+outputs within 1e-4 (fp32) / 2e-2 (bf16)."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as ge
+from oracle import pop_oracle as po
+from paper_2602_06822_b200 import pop, workloads as wl
+from tests import parity as pr
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    ge.build()
+    pop.lib()
+
+
+def weights_dev(w):
+    return pr.to_dev(w.weights.Wg), pr.to_dev(w.weights.Wu), pr.to_dev(w.weights.Wd)
+
+
+def weights_host(w):
+    return tuple(np.asarray(a.values, dtype=np.float64) for a in (w.weights.Wg, w.weights.Wu, w.weights.Wd))
+
+
+def run_decode_parity(w, part, R, C, steps, k, Wh):
+    cfg = w.cfg
+    dev = torch.device("cuda:0")
+    mask = torch.empty(max(part.n_cand, 1), dtype=torch.uint8, device=dev)[:part.n_cand]
+    sel = torch.empty(max(k, 1), dtype=torch.int32, device=dev)[:k]
+    worst, swaps = 0.0, 0
+    for t in range(steps):
+        x = pr.to_dev(w.xs, index=t)
+        mask.fill_(7)
+        sel.fill_(-1)
+        y = pop.decode_step(part, x, k, mask_out=mask, sel_out=sel)
+        torch.cuda.synchronize()
+        o = po.decode_step(w.xs.values[t], *Wh, R, C, k)
+        m, s = mask.cpu().numpy(), sel.cpu().numpy()
+        sw = pr.check_selection(s, m, C, o, k)
+        yref = o["y"]
+        if sw:   # an allowed near-tie swap: compare y with the oracle run under the GPU's mask
+            active = np.sort(np.concatenate([R, s]))
+            yref = po.masked_ffn(w.xs.values[t], *Wh, active)
+        swaps += sw
+        worst = max(worst, pr.rel_err(pr.host_values(y), yref))
+    part.check()
+    assert worst <= pr.TOL[cfg.dtype], f"max relative output error {worst:.3e}"
+    return worst, swaps
+
+
+def run_case(cfg, steps=None, k=None, check_scores=True):
+    w = wl.make_ffn_workload(cfg, steps)
+    steps = w.xs.values.shape[0]
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, cfg.ratios.astuple())
+    ref = po.prefill_partition(w.X.values, *Wh, cfg.ratios.astuple())
+    assert (part.n_ret, part.n_cand, part.n_pruned) == (ref["R"].size, ref["C"].size, ref["P"].size)
+    if check_scores:
+        np.testing.assert_allclose(part.scores(), ref["scores"], rtol=1e-9, atol=1e-300)
+    pr.check_regions(part, ref)
+    R, C, _ = part.indices()
+    if k is None:
+        k = cfg.k if cfg.k is not None else part.n_cand // 2
+    out = run_decode_parity(w, part, R, C, steps, k, Wh)
+    part.destroy()
+    return out
+
+
+# ------------------------------------------------------------------ config 1 (full, fp32)
+def test_config1_full():
+    cfg = wl.config1()
+    assert pop.region_sizes(cfg.N, cfg.ratios.astuple()) == (414, 550, 412, 275)
+    run_case(cfg)
+
+
+# ------------------------------------------------------------------ small shapes, several tiles + ragged tails
+@pytest.mark.parametrize("d,N,L,B,dtype", [
+    (256, 640, 40, 1, wl.BF16),
+    (264, 1000, 33, 1, wl.BF16),      # d not a multiple of 256; N, L ragged
+    (1024, 1111, 70, 2, wl.BF16),
+    (512, 777, 65, 3, wl.BF16),
+    (320, 900, 20, 8, wl.BF16),
+    (100, 333, 19, 1, wl.F32),
+    (768, 1500, 50, 4, wl.F32),
+])
+def test_small_shapes(d, N, L, B, dtype):
+    cfg = wl.FFNConfig(f"s{d}x{N}", d=d, N=N, dtype=dtype, prompt_tokens=L, decode_steps=5, batch=B,
+                       ratios=wl.Ratios(0.45, 0.25, 0.30), seed=d + N)
+    run_case(cfg)
+
+
+# ------------------------------------------------------------------ degenerate settings
+@pytest.mark.parametrize("ratios,kfrac", [
+    ((1.0, 0.0, 0.0), 0.0),     # nothing pruned: dense FFN
+    ((0.0, 1.0, 0.0), 0.6),     # every channel a candidate (ablation Variant (2))
+    ((0.0, 0.5, 0.5), 0.5),     # no retained channels
+    ((0.5, 0.0, 0.5), 0.0),     # no candidates: static mask
+    ((0.4, 0.3, 0.3), 0.0),     # k = 0
+    ((0.4, 0.3, 0.3), 1.0),     # k = n_C
+])
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_degenerate_regions(ratios, kfrac, dtype):
+    cfg = wl.FFNConfig("deg", d=256, N=500, dtype=dtype, prompt_tokens=24, decode_steps=3, batch=2,
+                       ratios=wl.Ratios(*ratios), seed=17)
+    n_C = po.region_sizes(cfg.N, ratios)[1]
+    run_case(cfg, k=int(round(kfrac * n_C)))
+
+
+def test_zero_pruning_equals_dense_ffn_on_gpu():
+    cfg = wl.FFNConfig("dense", d=512, N=1376, dtype=wl.F32, prompt_tokens=16, decode_steps=2, batch=1,
+                       ratios=wl.Ratios(1.0, 0.0, 0.0), seed=3)
+    w = wl.make_ffn_workload(cfg)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, (1.0, 0.0, 0.0))
+    x = pr.to_dev(w.xs, index=0)
+    y = pop.decode_step(part, x, 0)
+    ref = torch.nn.functional.linear(
+        torch.nn.functional.silu(torch.nn.functional.linear(x.double(), Wg.double()))
+        * torch.nn.functional.linear(x.double(), Wu.double()), Wd.double())
+    assert pr.rel_err(pr.host_values(y), ref.cpu().numpy()) <= 1e-4
+    part.destroy()
+
+
+def test_exact_ties_break_by_lower_channel_index():
+    w = wl.make_tie_case()
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, w.cfg.ratios.astuple())
+    ref = po.prefill_partition(w.X.values, *Wh, w.cfg.ratios.astuple())
+    R, C, P = part.indices()
+    # exact equality, no allowance: duplicated channels have bit-equal scores on both sides
+    assert np.array_equal(R, ref["R"]) and np.array_equal(C, ref["C"]) and np.array_equal(P, ref["P"])
+    sc = part.scores()
+    assert sc[1] == sc[5] == sc[9] and sc[0] == 0.0 and sc[13] == 0.0
+    part.destroy()
+    # decode ties: make every channel a candidate so the duplicated channels compete directly
+    ret = np.array([3, 4], dtype=np.int32)
+    cand = np.array([i for i in range(w.cfg.N) if i not in (3, 4, 40)], dtype=np.int32)
+    part = pop.partition_from_indices(Wg, Wu, Wd, ret, cand)
+    for k in (0, 1, 7, 20, cand.size - 1, cand.size):
+        mask = torch.zeros(cand.size, dtype=torch.uint8, device="cuda:0")
+        sel = torch.zeros(max(k, 1), dtype=torch.int32, device="cuda:0")[:k]
+        for t in range(w.xs.values.shape[0]):
+            y = pop.decode_step(part, pr.to_dev(w.xs, index=t), k, mask_out=mask, sel_out=sel)
+            o = po.decode_step(w.xs.values[t], *Wh, ret, cand, k)
+            assert np.array_equal(sel.cpu().numpy(), o["sel"])
+            assert np.array_equal(mask.cpu().numpy(), o["mask"])
+            assert pr.rel_err(pr.host_values(y), o["y"]) <= 1e-4
+    part.check()
+    part.destroy()
+
+
+def test_partition_from_indices_and_argument_errors():
+    cfg = wl.FFNConfig("fi", d=128, N=200, dtype=wl.BF16, prompt_tokens=8, decode_steps=2, seed=21)
+    w = wl.make_ffn_workload(cfg)
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    rng = np.random.default_rng(0)
+    perm = rng.permutation(200)
+    ret, cand = np.sort(perm[:90]).astype(np.int32), np.sort(perm[90:150]).astype(np.int32)
+    part = pop.partition_from_indices(Wg, Wu, Wd, ret, cand)
+    R, C, P = part.indices()
+    assert np.array_equal(R, ret) and np.array_equal(C, cand) and np.array_equal(P, np.sort(perm[150:]))
+    run_decode_parity(w, part, R, C, 2, 30, Wh)
+    x = pr.to_dev(w.xs, index=0)
+    for bad_k in (-1, 61):
+        with pytest.raises(pop.PopError) as e:
+            pop.decode_step(part, x, bad_k)
+        assert e.value.status == pop.POP_ERR_INVALID_ARG
+    with pytest.raises(pop.PopError) as e:
+        pop.decode_step(part, torch.zeros(9, 128, dtype=torch.bfloat16, device="cuda:0"), 3)
+    assert e.value.status == pop.POP_ERR_UNSUPPORTED
+    part.destroy()
+    for bad in ((np.array([5, 3], np.int32), cand), (np.array([1, 1], np.int32), cand),
+                (np.array([cand[0]], np.int32), cand), (np.array([200], np.int32), cand)):
+        with pytest.raises(pop.PopError) as e:
+            pop.partition_from_indices(Wg, Wu, Wd, *bad)
+        assert e.value.status == pop.POP_ERR_INVALID_ARG
+    with pytest.raises(pop.PopError) as e:
+        pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, (0.5, 0.6, 0.6))
+    assert e.value.status == pop.POP_ERR_INVALID_ARG
+
+
+def test_repeated_steps_are_bit_identical_in_mask_and_close_in_output():
+    cfg = wl.FFNConfig("rep", d=512, N=1024, dtype=wl.BF16, prompt_tokens=32, decode_steps=1, seed=5)
+    w = wl.make_ffn_workload(cfg)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, (0.5, 0.3, 0.2))
+    x = pr.to_dev(w.xs, index=0)
+    k = part.n_cand // 2
+    m1 = torch.zeros(part.n_cand, dtype=torch.uint8, device="cuda:0")
+    m2 = torch.zeros_like(m1)
+    y1 = pop.decode_step(part, x, k, mask_out=m1).clone()
+    y2 = pop.decode_step(part, x, k, mask_out=m2).clone()
+    assert torch.equal(m1, m2)
+    assert pr.rel_err(pr.host_values(y2), pr.host_values(y1)) <= 1e-2
+    part.destroy()
+
+
+# ------------------------------------------------------------------ full-size workloads
+@pytest.mark.parametrize("r", [0.2, 0.4])
+def test_config2_full_size(r):
+    cfg = wl.config2(r)
+    assert po.region_sizes(cfg.N, cfg.ratios.astuple())[:2] == ((8257, 1100) if r == 0.2 else (6056, 1100))
+    run_case(cfg, steps=6)
+
+
+@pytest.mark.parametrize("batch", [1, 8])
+def test_config5_full_size(batch):
+    cfg = wl.config5(batch)
+    run_case(cfg, steps=3)
