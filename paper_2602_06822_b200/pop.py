@@ -120,7 +120,7 @@ class _DevView:
     """Minimal __cuda_array_interface__ carrier for a raw device pointer."""
 
     def __init__(self, ptr: int, n: int, typestr: str):
-        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (int(ptr), True),
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (int(ptr), False),
                                          "version": 2, "strides": None}
 
 
