@@ -53,6 +53,10 @@ const char* pop_status_string(int status);
 /* Text of the last CUDA runtime error seen by this thread inside the library ("" if none). */
 const char* pop_last_cuda_error(void);
 
+/* Number of CUDA kernels this library has launched in this process so far (kernels recorded into
+ * a CUDA graph during stream capture count once, at capture). */
+unsigned long long pop_kernel_launch_count(void);
+
 /*
  * Region sizes for N channels (Sec. 3.3: thresholds at the (r - delta) and (r + delta) quantiles;
  * taken by rank so that the sizes are exact):

@@ -13,6 +13,10 @@ void pop_set_cuda_error(cudaError_t e, const char* what) {
     (void)cudaGetLastError();   // clear the sticky-free error state
 }
 
+static unsigned long long g_launches = 0;
+void pop_count_launch(int n) { __atomic_fetch_add(&g_launches, (unsigned long long)n, __ATOMIC_RELAXED); }
+extern "C" unsigned long long pop_kernel_launch_count(void) { return __atomic_load_n(&g_launches, __ATOMIC_RELAXED); }
+
 extern "C" const char* pop_version(void) { return "pop-b200 0.1.0 (sm_100a)"; }
 
 extern "C" const char* pop_last_cuda_error(void) { return g_cuda_err; }

@@ -61,6 +61,15 @@ void pop_set_cuda_error(cudaError_t e, const char* what);
         }                                                                 \
     } while (0)
 
+// Every kernel launch of the library goes through POP_LAUNCHED() so that callers can report
+// how many of the library's kernels ran (pop_kernel_launch_count()).
+void pop_count_launch(int n);
+#define POP_LAUNCHED()                         \
+    do {                                       \
+        POP_CUDA(cudaGetLastError());          \
+        pop_count_launch(1);                   \
+    } while (0)
+
 // ---------------------------------------------------------------------------------------------
 // launchers implemented in the .cu files (host functions; all enqueue on `st`)
 // ---------------------------------------------------------------------------------------------

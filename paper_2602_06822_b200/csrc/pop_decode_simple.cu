@@ -138,21 +138,21 @@ static int decode_simple_t(pop_partition* p, const void* x, int B, int k, void* 
     if (p->n_rc > 0) {
         gateup_simple_kernel<T><<<(p->n_rc + 7) / 8, 256, 0, st>>>((const uint4*)p->GU, (const uint4*)x, B, row_vecs,
                                                                   p->n_ret, p->n_rc, p->norm_cand, p->h, p->keys);
-        POP_CUDA(cudaGetLastError());
+        POP_LAUNCHED();
     }
     if (p->n_cand > 0) {
         select_simple_kernel<<<1, SEL_NT, 0, st>>>(p->keys, p->n_cand, k, p->idx_cand, p->sel_slots, mask_out, sel_out);
-        POP_CUDA(cudaGetLastError());
+        POP_LAUNCHED();
     }
     const int n_act = p->n_ret + k;
     if (n_act > 0) {
         const int rpb = 16;
         down_simple_kernel<T><<<(n_act + rpb - 1) / rpb, 256, 0, st>>>((const uint4*)p->WdT, p->h, p->sel_slots, B, p->d,
                                                                        row_vecs, p->n_ret, p->n_rc, k, rpb, p->y_acc);
-        POP_CUDA(cudaGetLastError());
+        POP_LAUNCHED();
     }
     finalize_simple_kernel<T><<<(B * p->d + 255) / 256, 256, 0, st>>>(p->y_acc, (T*)y, B * p->d);
-    POP_CUDA(cudaGetLastError());
+    POP_LAUNCHED();
     return POP_OK;
 }
 

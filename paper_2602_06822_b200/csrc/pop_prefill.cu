@@ -36,7 +36,7 @@ int pop_launch_colnorm(const void* Wd, int d, int N, pop_dtype_t dt, double* nor
     dim3 blk(32, 32), grd((N + 31) / 32);
     if (dt == POP_F32) colnorm_kernel<float><<<grd, blk, 0, st>>>((const float*)Wd, d, N, norm);
     else colnorm_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, d, N, norm);
-    POP_CUDA(cudaGetLastError());
+    POP_LAUNCHED();
     return POP_OK;
 }
 
@@ -130,7 +130,7 @@ int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, con
         prefill_s2_exact_kernel<__nv_bfloat16><<<grd, 256, 0, st>>>(
             (const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, N,
             chan_list, n_list, s2);
-    POP_CUDA(cudaGetLastError());
+    POP_LAUNCHED();
     return POP_OK;
 }
 
@@ -143,7 +143,7 @@ __global__ void scores_kernel(const double* __restrict__ s2, const double* __res
 
 int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st) {
     scores_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2, norm, N, scores);
-    POP_CUDA(cudaGetLastError());
+    POP_LAUNCHED();
     return POP_OK;
 }
 
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(PART_NT) partition_kernel(const double* __rest
 int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* idx_ret,
                          int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st) {
     partition_kernel<<<1, PART_NT, 0, st>>>(scores, N, n_ret, n_cand, idx_ret, idx_cand, idx_pruned);
-    POP_CUDA(cudaGetLastError());
+    POP_LAUNCHED();
     return POP_OK;
 }
 
@@ -258,7 +258,7 @@ int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, co
         const int row_vecs = p->d * p->es / 16;
         repack_gu_kernel<<<p->n_rc, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, p->n_ret,
                                                   p->idx_ret, p->idx_cand, (uint4*)p->GU);
-        POP_CUDA(cudaGetLastError());
+        POP_LAUNCHED();
         dim3 blk(32, 32), grd((p->n_rc + 31) / 32, (p->d + 31) / 32);
         if (p->dtype == POP_F32)
             repack_wdt_kernel<float><<<grd, blk, 0, st>>>((const float*)Wd, p->d, p->N, p->n_rc, p->n_ret,
@@ -267,11 +267,11 @@ int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, co
             repack_wdt_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_rc,
                                                                    p->n_ret, p->idx_ret, p->idx_cand,
                                                                    (__nv_bfloat16*)p->WdT);
-        POP_CUDA(cudaGetLastError());
+        POP_LAUNCHED();
     }
     if (p->n_cand > 0) {
         gather_norm_kernel<<<(p->n_cand + 255) / 256, 256, 0, st>>>(norm, p->idx_cand, p->n_cand, p->norm_cand);
-        POP_CUDA(cudaGetLastError());
+        POP_LAUNCHED();
     }
     return POP_OK;
 }

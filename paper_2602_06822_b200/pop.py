@@ -45,6 +45,7 @@ SIGNATURES = {
     "pop_version": (C.c_char_p, []),
     "pop_status_string": (C.c_char_p, [C.c_int]),
     "pop_last_cuda_error": (C.c_char_p, []),
+    "pop_kernel_launch_count": (C.c_ulonglong, []),
     "pop_region_sizes": (C.c_int, [C.c_int, Ratios] + [C.POINTER(C.c_int)] * 4),
     "pop_prefill_partition": (C.c_int, [_P, C.c_int, C.c_int, _P, _P, _P, C.c_int, C.c_int, Ratios, _P,
                                         C.POINTER(_P)]),
@@ -76,6 +77,10 @@ def lib() -> C.CDLL:
 
 def version() -> str:
     return lib().pop_version().decode()
+
+
+def kernel_launch_count() -> int:
+    return int(lib().pop_kernel_launch_count())
 
 
 def status_string(status: int) -> str:
