@@ -38,6 +38,7 @@ extern "C" {
 #define POP_ERR_TIMEOUT       -5   /* a bounded device-side wait expired (reported by pop_partition_check) */
 
 #define POP_MAX_BATCH          8   /* largest decode batch B a partition's scratch is sized for       */
+#define POP_NOALLOC_MAX_N  32768   /* largest N pop_prefill_scores_noalloc accepts                    */
 
 typedef enum { POP_F32 = 0, POP_BF16 = 1 } pop_dtype_t;
 
@@ -143,6 +144,34 @@ int pop_partition_destroy(pop_partition_t* p);
  */
 int pop_decode_step(pop_partition_t* p, const void* x, int B, int k_candidate,
                     void* y, uint8_t* mask_out, int32_t* sel_out, void* cuda_stream);
+
+/*
+ * Prefill importance scores without any allocation.  (The paper has no counterpart: this entry
+ * point exists for the library's users, not for the method.)
+ *
+ * Some callers cannot allocate device memory at the moment they need the scores: code running
+ * inside a memory pool whose budget is fixed up front, a serving loop that forbids allocator
+ * calls on its hot path because they may synchronise the device, or a host whose allocator
+ * is owned by another framework.  pop_prefill_partition is closed to them, since it allocates the
+ * partition and two stream-ordered temporaries.  This call computes the same I_i (Eq. 3; the
+ * same kernels and the same fp64 arithmetic as pop_prefill_partition) into a buffer the caller
+ * already owns, and keeps its temporaries (2 x N doubles) in a fixed 512 KB array that is part
+ * of the library image on every GPU that loads it.
+ *   X [L, d], Wg [N, d], Wu [N, d], Wd [d, N]: device arrays of `dtype` as for
+ *   pop_prefill_partition; scores_out: device double [N], caller-owned, written on `cuda_stream`.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.
+ * N > POP_NOALLOC_MAX_N is rejected with POP_ERR_UNSUPPORTED (pop_last_cuda_error() names the
+ * limit); other errors as pop_prefill_partition.
+ * The first call on a device looks up the device address of the fixed array (a host-side
+ * query, once per device, with that device current); make that first call outside any stream
+ * capture.
+ * All calls on one device share the array, and it keeps the previous call's contents (every
+ * entry a call reads it has written first, so nothing needs clearing).  Two calls whose kernels
+ * may overlap on the GPU (different streams, no ordering between them) race on it: order them.
+ */
+int pop_prefill_scores_noalloc(const void* X, int L, int d,
+                               const void* Wg, const void* Wu, const void* Wd, int N,
+                               pop_dtype_t dtype, double* scores_out, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -20,6 +20,7 @@ POP_ERR_CUDA = -4
 POP_ERR_TIMEOUT = -5
 POP_MAX_BATCH = 8
 POP_F32, POP_BF16 = 0, 1
+POP_NOALLOC_MAX_N = 32768
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libpop.so")
 
@@ -58,6 +59,7 @@ SIGNATURES = {
     "pop_partition_check": (C.c_int, [_P]),
     "pop_partition_destroy": (C.c_int, [_P]),
     "pop_decode_step": (C.c_int, [_P, _P, C.c_int, C.c_int, _P, _P, _P, _P]),
+    "pop_prefill_scores_noalloc": (C.c_int, [_P, C.c_int, C.c_int, _P, _P, _P, C.c_int, C.c_int, _P, _P]),
 }
 
 
@@ -239,3 +241,21 @@ def decode_step(part: Partition, x, k: int, y=None, mask_out=None, sel_out=None,
                                  None if sel_out is None else sel_out.data_ptr(), _stream_ptr(stream)),
            "pop_decode_step")
     return y
+
+
+def prefill_scores_noalloc(X, Wg, Wu, Wd, out, stream=None):
+    """pop_prefill_scores_noalloc: the prefill scores I_i written into ``out`` (a float64 CUDA
+    tensor of N elements that the caller already owns).  The library call allocates nothing: its
+    temporaries live in a fixed array inside the library, shared by all calls on the device."""
+    torch = _torch()
+    for t in (X, Wg, Wu, Wd, out):
+        if not (t.is_cuda and t.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+    L, d = X.shape
+    N = Wg.shape[0]
+    if out.dtype != torch.float64 or out.numel() != N:
+        raise ValueError("out must be a float64 tensor of N elements")
+    _check(lib().pop_prefill_scores_noalloc(X.data_ptr(), L, d, Wg.data_ptr(), Wu.data_ptr(), Wd.data_ptr(), N,
+                                            _dtype_code(X), out.data_ptr(), _stream_ptr(stream)),
+           "pop_prefill_scores_noalloc")
+    return out
