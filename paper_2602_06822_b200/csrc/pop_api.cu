@@ -72,7 +72,7 @@ static void partition_free(pop_partition* p) {
     if (!p) return;
     cudaFree(p->GU); cudaFree(p->WdT); cudaFree(p->idx_ret); cudaFree(p->idx_cand); cudaFree(p->idx_pruned);
     cudaFree(p->scores); cudaFree(p->norm_cand); cudaFree(p->h); cudaFree(p->keys); cudaFree(p->y_acc);
-    cudaFree(p->sel_slots); cudaFree(p->sync);
+    cudaFree(p->sel_slots); cudaFree(p->sync); cudaFree(p->flags);
     free(p);
 }
 
@@ -89,23 +89,40 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device);
     cudaDeviceGetAttribute(&p->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
     const size_t row = (size_t)d * p->es;
+    // bf16 shapes the streaming decode kernel takes get the tiled layout (POP_DECODE_IMPL=fused or
+    // =simple keeps the row layout and the older kernels, for comparison)
+    const char* impl = getenv("POP_DECODE_IMPL");
+    const bool force_rows = impl && (!strcmp(impl, "fused") || !strcmp(impl, "simple"));
+    p->layout = (!force_rows && pop_stream_layout_supported(d, dt)) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
+    p->n_rt = (n_ret + 7) / 8;
+    p->n_cg = (n_ret + 15) / 16;
+    p->n_ret_pad = 16 * p->n_cg;
+    p->h_stride = p->layout == POP_LAYOUT_TILED ? p->n_ret_pad + ((n_cand + 15) / 16) * 16 : (p->n_rc > 0 ? p->n_rc : 1);
 #define TRY(x) do { rc = (x); if (rc != POP_OK) { partition_free(p); return rc; } } while (0)
-    TRY(dev_alloc(&p->GU, (size_t)p->n_rc * 2 * row));
-    TRY(dev_alloc(&p->WdT, (size_t)p->n_rc * row));
+    if (p->layout == POP_LAYOUT_TILED) {
+        TRY(dev_alloc(&p->GU, ((size_t)p->n_rt * 16 + (size_t)n_cand * 2) * row));
+        TRY(dev_alloc(&p->WdT, ((size_t)p->n_ret_pad + (size_t)n_cand) * row));
+    } else {
+        TRY(dev_alloc(&p->GU, (size_t)p->n_rc * 2 * row));
+        TRY(dev_alloc(&p->WdT, (size_t)p->n_rc * row));
+    }
     TRY(dev_alloc(&p->idx_ret, sizeof(int32_t) * (size_t)n_ret));
     TRY(dev_alloc(&p->idx_cand, sizeof(int32_t) * (size_t)n_cand));
     TRY(dev_alloc(&p->idx_pruned, sizeof(int32_t) * (size_t)p->n_pruned));
     TRY(dev_alloc(&p->scores, sizeof(double) * (size_t)N));
     TRY(dev_alloc(&p->norm_cand, sizeof(double) * (size_t)n_cand));
-    TRY(dev_alloc(&p->h, sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->n_rc > 0 ? p->n_rc : 1)));
+    TRY(dev_alloc(&p->h, sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1)));
     TRY(dev_alloc(&p->keys, sizeof(u64) * (size_t)n_cand));
     TRY(dev_alloc(&p->y_acc, sizeof(float) * (size_t)POP_MAX_BATCH * d));
     TRY(dev_alloc(&p->sel_slots, sizeof(int32_t) * (size_t)n_cand));
     TRY(dev_alloc(&p->sync, sizeof(u32) * SYNC_WORDS));
+    TRY(dev_alloc(&p->flags, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1)));
 #undef TRY
     e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->scores, 0, sizeof(double) * (size_t)N, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->flags, 0, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1), st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1), st);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free(p); return POP_ERR_CUDA; }
     *out = p;
     return POP_OK;
@@ -143,7 +160,8 @@ extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg
     if (rc == POP_OK) rc = pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
     if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, p->scores, st);
     if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->idx_ret, p->idx_cand, p->idx_pruned, st);
-    if (rc == POP_OK) rc = pop_launch_repack(p, Wg, Wu, Wd, norm, st);
+    if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
+                                                         : pop_launch_repack(p, Wg, Wu, Wd, norm, st);
     cudaFreeAsync(norm, st);
     cudaFreeAsync(s2, st);
     if (rc != POP_OK) { cudaStreamSynchronize(st); partition_free(p); return rc; }
@@ -200,7 +218,8 @@ extern "C" int pop_partition_from_indices(const void* Wg, const void* Wu, const 
     e = cudaMallocAsync((void**)&norm, sizeof(double) * (size_t)N, st);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMallocAsync"); partition_free(p); return POP_ERR_ALLOC; }
     rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
-    if (rc == POP_OK) rc = pop_launch_repack(p, Wg, Wu, Wd, norm, st);
+    if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
+                                                         : pop_launch_repack(p, Wg, Wu, Wd, norm, st);
     cudaFreeAsync(norm, st);
     if (rc != POP_OK) { cudaStreamSynchronize(st); partition_free(p); return rc; }
     *out = p;
@@ -244,9 +263,11 @@ extern "C" int pop_partition_check(pop_partition_t* p) {
     u32 flag = 0;
     POP_CUDA(cudaMemcpy(&flag, p->sync + SYNC_ERROR, sizeof(u32), cudaMemcpyDeviceToHost));
     if (flag) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "a bounded device-side wait expired in a decode step (wait code %u)", flag);
         // leave the partition usable: clear counters and the accumulator
         POP_CUDA(cudaMemset(p->sync, 0, sizeof(u32) * SYNC_WORDS));
         POP_CUDA(cudaMemset(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * p->d));
+        POP_CUDA(cudaMemset(p->flags, 0, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1)));
         return POP_ERR_TIMEOUT;
     }
     return POP_OK;
@@ -265,6 +286,7 @@ extern "C" int pop_decode_step(pop_partition_t* p, const void* x, int B, int k_c
     if (B > POP_MAX_BATCH) return POP_ERR_UNSUPPORTED;
     if (!aligned16(x) || !aligned16(y)) return POP_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (p->layout == POP_LAYOUT_TILED) return pop_launch_decode_stream(p, x, B, k_candidate, y, mask_out, sel_out, st);
     int rc = pop_launch_decode(p, x, B, k_candidate, y, mask_out, sel_out, st);
     if (rc == POP_ERR_UNSUPPORTED) rc = pop_launch_decode_simple(p, x, B, k_candidate, y, mask_out, sel_out, st);
     return rc;

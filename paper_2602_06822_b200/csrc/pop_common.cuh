@@ -15,15 +15,35 @@ typedef unsigned int u32;
 //
 // Repacked layout ("slots"): slot s in [0, n_ret) is Retained channel idx_ret[s]; slot
 // n_ret + c is Candidate channel idx_cand[c].  n_rc = n_ret + n_cand.
+//
+// POP_LAYOUT_ROWS (any dtype and shape)
 //   GU  [n_rc][2][d]  gate row then up row of the slot's channel, contiguous (one 2*d*es block)
 //   WdT [n_rc][d]     column of the down projection of the slot's channel, as a contiguous row
+//   h   [POP_MAX_BATCH][n_rc]
+//
+// POP_LAYOUT_TILED (bf16, d a multiple of 1024; read by pop_decode_stream.cu).  The Retained part
+// is stored as mma.m16n8k16 A fragments, 512 bytes per (16 x 16) tile, lane L's 16 bytes =
+// {A[g][2t..2t+1], A[g+8][2t..], A[g][2t+8..], A[g+8][2t+8..]} with g = L / 4, t = L % 4:
+//   GU  = GUt  [n_rt][d/16][32][16 B]      tile (rt, kt): rows 0..7 gate, rows 8..15 up of retained
+//                                            slots 8 rt .. 8 rt + 7, columns = hidden 16 kt .. 16 kt + 15
+//         GUc  [n_cand][2][d]              candidate gate/up rows, plain
+//   WdT = WdTt [4][n_cg][d/64][32][16 B]   tile (q, cg, mt): rows = outputs q d/4 + 16 mt .. + 15,
+//                                            columns = retained slots 16 cg .. 16 cg + 15
+//         WdTc [n_cand][d]                 candidate down rows, plain
+//   n_rt = ceil(n_ret / 8), n_cg = ceil(n_ret / 16), n_ret_pad = 16 n_cg; slots past n_ret are zero.
+//   h   [POP_MAX_BATCH][h_stride]: retained slots at [0, n_ret_pad) (padding stays 0), candidates
+//       at n_ret_pad + c.
 // ---------------------------------------------------------------------------------------------
+enum { POP_LAYOUT_ROWS = 0, POP_LAYOUT_TILED = 1 };
+
 struct pop_partition {
     int device;
     int d, N;
     pop_dtype_t dtype;
     int es;                       // element size in bytes
     int n_ret, n_cand, n_pruned, n_rc;
+    int layout;                   // POP_LAYOUT_*
+    int n_rt, n_cg, n_ret_pad, h_stride;      // tiled layout only (h_stride: both)
 
     void* GU;
     void* WdT;
@@ -38,14 +58,17 @@ struct pop_partition {
     u64* keys;                    // [n_cand] candidate scores as ordered 64-bit keys
     float* y_acc;                 // [POP_MAX_BATCH][d] fp32 accumulator, zero between steps
     int32_t* sel_slots;           // [n_cand] selected candidate slots (ascending), this step
-    u32* sync;                    // [16] counters / flags, see pop_decode.cu
+    u32* sync;                    // [SYNC_WORDS] counters / flags, see pop_decode*.cu
+    u32* flags;                   // [n_rt] tiled layout: epoch at which a phase-1 unit published its h
     int sm_count;
     int coop;                     // device supports cooperative launch
     int max_smem_optin;
 };
 
-// sync[] word assignment
-enum { SYNC_BARRIER = 0, SYNC_TICKET = 1, SYNC_ERROR = 2, SYNC_WORK = 3, SYNC_WORDS = 16 };
+// sync[] word assignment (contended counters sit on separate 128-byte lines)
+enum { SYNC_BARRIER = 0, SYNC_TICKET = 1, SYNC_ERROR = 2, SYNC_WORK = 3,
+       SYNC_EPOCH = 32, SYNC_SEL_READY = 33, SYNC_P1 = 64, SYNC_CAND_DONE = 96,
+       SYNC_Q0 = 128 /* + 32 q, q = 0..3 */, SYNC_WORDS = 256 };
 
 // ---------------------------------------------------------------------------------------------
 // error plumbing
@@ -83,6 +106,12 @@ int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand,
                          int32_t* idx_ret, int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);
 int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                       const double* norm /*[N]*/, cudaStream_t st);
+int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
+                            const double* norm /*[N]*/, cudaStream_t st);
+// pop_decode_stream.cu (bf16 partitions in the tiled layout)
+bool pop_stream_layout_supported(int d, pop_dtype_t dt);
+int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void* y,
+                             uint8_t* mask_out, int32_t* sel_out, cudaStream_t st);
 // pop_decode_simple.cu (multi-kernel path, any accepted shape)
 int pop_launch_decode_simple(pop_partition* p, const void* x, int B, int k, void* y,
                              uint8_t* mask_out, int32_t* sel_out, cudaStream_t st);

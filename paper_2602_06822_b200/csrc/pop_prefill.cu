@@ -275,3 +275,95 @@ int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, co
     }
     return POP_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Repack into the tiled layout (see pop_common.cuh): the Retained rows as mma.m16n8k16 A
+// fragments, the Candidate rows plain.  One thread writes one 16-byte fragment piece.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) repack_gut_kernel(const __nv_bfloat16* __restrict__ Wg,
+                                                         const __nv_bfloat16* __restrict__ Wu, int d, int n_ret,
+                                                         int n_rt, const int32_t* __restrict__ idx_ret,
+                                                         uint4* __restrict__ GUt) {
+    const int KT = d >> 4;
+    const size_t total = (size_t)n_rt * KT * 32;
+    for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (size_t)gridDim.x * blockDim.x) {
+        const int lane = (int)(o & 31);
+        const size_t tile = o >> 5;
+        const int kt = (int)(tile % KT), rt = (int)(tile / KT);
+        const int g = lane >> 2, t = lane & 3;
+        const int slot = 8 * rt + g;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (slot < n_ret) {
+            const int ch = idx_ret[slot];
+            const u32* gp = reinterpret_cast<const u32*>(Wg + (size_t)ch * d + (size_t)kt * 16);
+            const u32* up = reinterpret_cast<const u32*>(Wu + (size_t)ch * d + (size_t)kt * 16);
+            v.x = gp[t];        // row g     (gate), columns 2t, 2t+1
+            v.y = up[t];        // row g + 8 (up),   columns 2t, 2t+1
+            v.z = gp[t + 4];    // row g,     columns 2t+8, 2t+9
+            v.w = up[t + 4];    // row g + 8, columns 2t+8, 2t+9
+        }
+        GUt[o] = v;
+    }
+}
+
+__global__ void __launch_bounds__(256) repack_wdtt_kernel(const __nv_bfloat16* __restrict__ Wd, int d, int N,
+                                                          int n_ret, int n_cg, const int32_t* __restrict__ idx_ret,
+                                                          uint4* __restrict__ WdTt) {
+    const int MT = d >> 6;                                   // m-tiles per quarter
+    const size_t total = (size_t)4 * n_cg * MT * 32;
+    const unsigned short* W = reinterpret_cast<const unsigned short*>(Wd);
+    for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (size_t)gridDim.x * blockDim.x) {
+        const int lane = (int)(o & 31);
+        size_t tile = o >> 5;
+        const int mt = (int)(tile % MT); tile /= MT;
+        const int cg = (int)(tile % n_cg);
+        const int q = (int)(tile / n_cg);
+        const int g = lane >> 2, t = lane & 3;
+        const int j0 = q * (d >> 2) + mt * 16 + g;           // output row of A rows g (and g + 8)
+        u32 r[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int j = j0 + ((e & 1) ? 8 : 0);
+            const int s0 = 16 * cg + 2 * t + ((e >> 1) ? 8 : 0);
+            u32 lo = 0, hi = 0;
+            if (s0 < n_ret) lo = W[(size_t)j * N + idx_ret[s0]];
+            if (s0 + 1 < n_ret) hi = W[(size_t)j * N + idx_ret[s0 + 1]];
+            r[e] = lo | (hi << 16);
+        }
+        WdTt[o] = make_uint4(r[0], r[1], r[2], r[3]);
+    }
+}
+
+int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
+                            const double* norm, cudaStream_t st) {
+    const size_t row = (size_t)p->d * 2;
+    unsigned char* GUt = (unsigned char*)p->GU;
+    unsigned char* GUc = GUt + (size_t)p->n_rt * 16 * row;
+    unsigned char* WdTt = (unsigned char*)p->WdT;
+    unsigned char* WdTc = WdTt + (size_t)p->n_ret_pad * row;
+    if (p->n_rt > 0) {
+        const size_t total = (size_t)p->n_rt * (p->d / 16) * 32;
+        const int blocks = (int)((total + 255) / 256 < 148 * 64 ? (total + 255) / 256 : 148 * 64);
+        repack_gut_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, p->d, p->n_ret,
+                                                  p->n_rt, p->idx_ret, (uint4*)GUt);
+        POP_LAUNCHED();
+        const size_t total2 = (size_t)4 * p->n_cg * (p->d / 64) * 32;
+        const int blocks2 = (int)((total2 + 255) / 256 < 148 * 64 ? (total2 + 255) / 256 : 148 * 64);
+        repack_wdtt_kernel<<<blocks2, 256, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_ret, p->n_cg,
+                                                    p->idx_ret, (uint4*)WdTt);
+        POP_LAUNCHED();
+    }
+    if (p->n_cand > 0) {
+        const int row_vecs = (int)(row / 16);
+        repack_gu_kernel<<<p->n_cand, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, 0, p->idx_cand,
+                                                    p->idx_cand, (uint4*)GUc);
+        POP_LAUNCHED();
+        dim3 blk(32, 32), grd((p->n_cand + 31) / 32, (p->d + 31) / 32);
+        repack_wdt_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_cand, 0,
+                                                               p->idx_cand, p->idx_cand, (__nv_bfloat16*)WdTc);
+        POP_LAUNCHED();
+        gather_norm_kernel<<<(p->n_cand + 255) / 256, 256, 0, st>>>(norm, p->idx_cand, p->n_cand, p->norm_cand);
+        POP_LAUNCHED();
+    }
+    return POP_OK;
+}

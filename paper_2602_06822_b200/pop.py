@@ -33,7 +33,7 @@ class PopError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
         msg = f"{where}: {status_string(status)}"
-        if status in (POP_ERR_CUDA, POP_ERR_ALLOC):
+        if status in (POP_ERR_CUDA, POP_ERR_ALLOC, POP_ERR_TIMEOUT):
             msg += f" [{lib().pop_last_cuda_error().decode()}]"
         super().__init__(msg)
 

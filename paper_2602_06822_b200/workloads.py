@@ -226,16 +226,16 @@ def make_moe_workload(cfg: FFNConfig, n_experts: int = 8, top_k: int = 2,
 
 
 # --------------------------------------------------------------------------- adversarial small cases
-def make_tie_case(N: int = 48, d: int = 16, L: int = 8, seed: int = 7) -> FFNWorkload:
-    """A small fp32 layer with duplicated channels (exact score ties) and a few
+def make_tie_case(N: int = 48, d: int = 16, L: int = 8, seed: int = 7, dtype: str = F32) -> FFNWorkload:
+    """A small layer with duplicated channels (exact score ties) and a few
     all-zero channels (zero scores), to exercise the index tie-break."""
-    cfg = FFNConfig("ties", d=d, N=N, dtype=F32, prompt_tokens=L, decode_steps=4,
+    cfg = FFNConfig("ties", d=d, N=N, dtype=dtype, prompt_tokens=L, decode_steps=4,
                     ratios=Ratios(0.25, 0.5, 0.25), seed=seed)
-    w = make_weights(N, d, F32, seed)
+    w = make_weights(N, d, dtype, seed)
     Wg, Wu, Wd = (np.array(a.values) for a in (w.Wg, w.Wu, w.Wd))
     for src, dst in ((1, 5), (1, 9), (2, 30), (7, 8), (20, 41)):
         Wg[dst] = Wg[src]; Wu[dst] = Wu[src]; Wd[:, dst] = Wd[:, src]
     for z in (0, 13, 47):
         Wg[z] = 0.0
-    weights = FFNWeights(as_array(Wg, F32), as_array(Wu, F32), as_array(Wd, F32))
+    weights = FFNWeights(as_array(Wg, dtype), as_array(Wu, dtype), as_array(Wd, dtype))
     return FFNWorkload(cfg, weights, make_prefill_input(cfg), make_decode_inputs(cfg))
