@@ -72,7 +72,7 @@ static void partition_free(pop_partition* p) {
     if (!p) return;
     cudaFree(p->GU); cudaFree(p->WdT); cudaFree(p->idx_ret); cudaFree(p->idx_cand); cudaFree(p->idx_pruned);
     cudaFree(p->scores); cudaFree(p->norm_cand); cudaFree(p->h); cudaFree(p->keys); cudaFree(p->y_acc);
-    cudaFree(p->sel_slots); cudaFree(p->sync); cudaFree(p->flags);
+    cudaFree(p->sel_slots); cudaFree(p->sync); cudaFree(p->flags); cudaFree(p->wnorm_cand); cudaFree(p->margins); cudaFree(p->selflag); cudaFree(p->keys32); cudaFree(p->uexact); cudaFree(p->rpart);
     free(p);
 }
 
@@ -89,18 +89,20 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device);
     cudaDeviceGetAttribute(&p->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
     const size_t row = (size_t)d * p->es;
-    // bf16 shapes the streaming decode kernel takes get the tiled layout (POP_DECODE_IMPL=fused or
-    // =simple keeps the row layout and the older kernels, for comparison)
+    // POP_DECODE_IMPL (read at every partition creation) picks the decode kernel family: "stream" = tiled layout +
+    // the dataflow kernel of pop_decode_stream.cu for the bf16 shapes it takes (its one-warp selection holds up to
+    // 1536 candidate keys); anything else = row layout + the fused / simple kernels.
     const char* impl = getenv("POP_DECODE_IMPL");
-    const bool force_rows = impl && (!strcmp(impl, "fused") || !strcmp(impl, "simple"));
-    p->layout = (!force_rows && pop_stream_layout_supported(d, dt)) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
+    const bool want_stream = impl && !strcmp(impl, "stream");
+    p->layout = (want_stream && pop_stream_layout_supported(d, dt) && n_cand <= 1536) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
     p->n_rt = (n_ret + 7) / 8;
     p->n_cg = (n_ret + 15) / 16;
+    p->n_ct = (n_cand + 7) / 8;
     p->n_ret_pad = 16 * p->n_cg;
     p->h_stride = p->layout == POP_LAYOUT_TILED ? p->n_ret_pad + ((n_cand + 15) / 16) * 16 : (p->n_rc > 0 ? p->n_rc : 1);
 #define TRY(x) do { rc = (x); if (rc != POP_OK) { partition_free(p); return rc; } } while (0)
     if (p->layout == POP_LAYOUT_TILED) {
-        TRY(dev_alloc(&p->GU, ((size_t)p->n_rt * 16 + (size_t)n_cand * 2) * row));
+        TRY(dev_alloc(&p->GU, ((size_t)(p->n_rt + p->n_ct) * 16 + (size_t)n_cand * 2) * row));
         TRY(dev_alloc(&p->WdT, ((size_t)p->n_ret_pad + (size_t)n_cand) * row));
     } else {
         TRY(dev_alloc(&p->GU, (size_t)p->n_rc * 2 * row));
@@ -117,6 +119,12 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     TRY(dev_alloc(&p->sel_slots, sizeof(int32_t) * (size_t)n_cand));
     TRY(dev_alloc(&p->sync, sizeof(u32) * SYNC_WORDS));
     TRY(dev_alloc(&p->flags, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1)));
+    TRY(dev_alloc(&p->wnorm_cand, sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1)));
+    TRY(dev_alloc(&p->margins, sizeof(double) * (size_t)(n_cand > 0 ? n_cand : 1)));
+    TRY(dev_alloc(&p->selflag, (size_t)(n_cand > 0 ? n_cand : 1)));
+    TRY(dev_alloc(&p->keys32, sizeof(u32) * (size_t)(n_cand > 0 ? n_cand : 1)));
+    TRY(dev_alloc(&p->uexact, sizeof(u64) * (size_t)(n_cand > 0 ? n_cand : 1)));
+    TRY(dev_alloc(&p->rpart, sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1)));
 #undef TRY
     e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);

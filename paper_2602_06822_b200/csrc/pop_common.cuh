@@ -26,11 +26,13 @@ typedef unsigned int u32;
 // {A[g][2t..2t+1], A[g+8][2t..], A[g][2t+8..], A[g+8][2t+8..]} with g = L / 4, t = L % 4:
 //   GU  = GUt  [n_rt][d/16][32][16 B]      tile (rt, kt): rows 0..7 gate, rows 8..15 up of retained
 //                                            slots 8 rt .. 8 rt + 7, columns = hidden 16 kt .. 16 kt + 15
-//         GUc  [n_cand][2][d]              candidate gate/up rows, plain
+//                                            tiles n_rt .. n_rt + n_ct - 1 hold the candidate slots the same way
+//         GUc  [n_cand][2][d]              candidate gate/up rows, plain (read only to re-score exactly)
 //   WdT = WdTt [4][n_cg][d/64][32][16 B]   tile (q, cg, mt): rows = outputs q d/4 + 16 mt .. + 15,
 //                                            columns = retained slots 16 cg .. 16 cg + 15
 //         WdTc [n_cand][d]                 candidate down rows, plain
-//   n_rt = ceil(n_ret / 8), n_cg = ceil(n_ret / 16), n_ret_pad = 16 n_cg; slots past n_ret are zero.
+//   n_rt = ceil(n_ret / 8), n_ct = ceil(n_cand / 8), n_cg = ceil(n_ret / 16), n_ret_pad = 16 n_cg;
+//   slots past n_ret (n_cand) are zero.
 //   h   [POP_MAX_BATCH][h_stride]: retained slots at [0, n_ret_pad) (padding stays 0), candidates
 //       at n_ret_pad + c.
 // ---------------------------------------------------------------------------------------------
@@ -43,7 +45,7 @@ struct pop_partition {
     int es;                       // element size in bytes
     int n_ret, n_cand, n_pruned, n_rc;
     int layout;                   // POP_LAYOUT_*
-    int n_rt, n_cg, n_ret_pad, h_stride;      // tiled layout only (h_stride: both)
+    int n_rt, n_ct, n_cg, n_ret_pad, h_stride;      // tiled layout only (h_stride: both)
 
     void* GU;
     void* WdT;
@@ -52,6 +54,12 @@ struct pop_partition {
     int32_t* idx_pruned;
     double* scores;               // [N] prefill I_i
     double* norm_cand;            // [n_cand] ||Wd[:, i]||_2 of the candidate channels
+    float* wnorm_cand;            // [2][n_cand] max |Wg[i][:]|, max |Wu[i][:]| of the candidate channels
+    double* margins;              // [n_cand] decode scratch: error bound of each approximate candidate score
+    uint8_t* selflag;             // [n_cand] decode scratch of the selection
+    u32* keys32;                  // [n_cand] decode scratch: fp32 copies of the streamed candidate scores
+    u64* uexact;                  // [n_cand] decode scratch: exact keys of re-scored candidates
+    double* rpart;                // [4 n_cand][POP_MAX_BATCH] decode scratch: partial dot products of re-scoring jobs
 
     // decode scratch (no allocation at decode time)
     float* h;                     // [POP_MAX_BATCH][n_rc] intermediate activations of this step

@@ -334,11 +334,29 @@ __global__ void __launch_bounds__(256) repack_wdtt_kernel(const __nv_bfloat16* _
     }
 }
 
+// wmax[0][c] = max |Wg[idx_cand[c]][:]|, wmax[1][c] = max |Wu[idx_cand[c]][:]|: with max |x| they bound any
+// single product of a candidate's dot products (used by the error bound of its streamed score).  One warp per row.
+__global__ void __launch_bounds__(256) rownorm_cand_kernel(const __nv_bfloat16* __restrict__ Wg,
+                                                           const __nv_bfloat16* __restrict__ Wu, int d, int n_cand,
+                                                           const int32_t* __restrict__ idx_cand,
+                                                           float* __restrict__ wmax) {
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (r >= 2 * n_cand) return;
+    const int which = r / n_cand, c = r - which * n_cand;
+    const __nv_bfloat16* row = (which ? Wu : Wg) + (size_t)idx_cand[c] * d;
+    float mx = 0.f;
+    for (int j = lane; j < d; j += 32) mx = fmaxf(mx, fabsf(__bfloat162float(row[j])));
+#pragma unroll
+    for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if (lane == 0) wmax[r] = mx;
+}
+
 int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                             const double* norm, cudaStream_t st) {
     const size_t row = (size_t)p->d * 2;
     unsigned char* GUt = (unsigned char*)p->GU;
-    unsigned char* GUc = GUt + (size_t)p->n_rt * 16 * row;
+    unsigned char* GUtc = GUt + (size_t)p->n_rt * 16 * row;            // candidate tiles
+    unsigned char* GUc = GUt + (size_t)(p->n_rt + p->n_ct) * 16 * row;  // candidate rows
     unsigned char* WdTt = (unsigned char*)p->WdT;
     unsigned char* WdTc = WdTt + (size_t)p->n_ret_pad * row;
     if (p->n_rt > 0) {
@@ -354,6 +372,14 @@ int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* 
         POP_LAUNCHED();
     }
     if (p->n_cand > 0) {
+        const size_t totalc = (size_t)p->n_ct * (p->d / 16) * 32;
+        const int blocksc = (int)((totalc + 255) / 256 < 148 * 64 ? (totalc + 255) / 256 : 148 * 64);
+        repack_gut_kernel<<<blocksc, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, p->d, p->n_cand,
+                                                   p->n_ct, p->idx_cand, (uint4*)GUtc);
+        POP_LAUNCHED();
+        rownorm_cand_kernel<<<(2 * p->n_cand + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu,
+                                                                      p->d, p->n_cand, p->idx_cand, p->wnorm_cand);
+        POP_LAUNCHED();
         const int row_vecs = (int)(row / 16);
         repack_gu_kernel<<<p->n_cand, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, 0, p->idx_cand,
                                                     p->idx_cand, (uint4*)GUc);

@@ -19,6 +19,14 @@ def _built():
     pop.lib()
 
 
+@pytest.fixture(autouse=True, params=["fused", "stream"])
+def decode_impl(request, monkeypatch):
+    """Every case runs with both decode kernel families (the choice is made when a partition is created;
+    shapes the streaming kernel does not take use the fused / simple kernels either way)."""
+    monkeypatch.setenv("POP_DECODE_IMPL", request.param)
+    return request.param
+
+
 def weights_dev(w):
     return pr.to_dev(w.weights.Wg), pr.to_dev(w.weights.Wu), pr.to_dev(w.weights.Wd)
 
