@@ -113,7 +113,8 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     TRY(dev_alloc(&p->idx_pruned, sizeof(int32_t) * (size_t)p->n_pruned));
     TRY(dev_alloc(&p->scores, sizeof(double) * (size_t)N));
     TRY(dev_alloc(&p->norm_cand, sizeof(double) * (size_t)n_cand));
-    TRY(dev_alloc(&p->h, sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1)));
+    // (tiled layout: 8 bytes per element, the value with the epoch of the step that wrote it)
+    TRY(dev_alloc(&p->h, 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1)));
     TRY(dev_alloc(&p->keys, sizeof(u64) * (size_t)n_cand));
     TRY(dev_alloc(&p->y_acc, sizeof(float) * (size_t)POP_MAX_BATCH * d));
     TRY(dev_alloc(&p->sel_slots, sizeof(int32_t) * (size_t)n_cand));
@@ -130,7 +131,7 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->scores, 0, sizeof(double) * (size_t)N, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->flags, 0, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1), st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1), st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1), st);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free(p); return POP_ERR_CUDA; }
     *out = p;
     return POP_OK;
@@ -276,6 +277,7 @@ extern "C" int pop_partition_check(pop_partition_t* p) {
         POP_CUDA(cudaMemset(p->sync, 0, sizeof(u32) * SYNC_WORDS));
         POP_CUDA(cudaMemset(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * p->d));
         POP_CUDA(cudaMemset(p->flags, 0, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1)));
+        POP_CUDA(cudaMemset(p->h, 0, 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1)));
         return POP_ERR_TIMEOUT;
     }
     return POP_OK;

@@ -157,7 +157,7 @@ __device__ __forceinline__ void warp_allreduce(double (&v)[NV]) {
 // chunks (of 32 lanes x 16 bytes) owned by each consumer warp.
 // ---------------------------------------------------------------------------------------------
 template <typename T, int BT, int CPW>
-__global__ void __launch_bounds__(544, 1) pop_decode_fused_kernel(const DecodeParams P) {
+__global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodeParams P) {
     constexpr int VEC = Elem<T>::VEC;
     constexpr int ES = (int)sizeof(T);
     constexpr bool IS_BF16 = (ES == 2);
@@ -630,7 +630,9 @@ int pop_launch_decode(pop_partition* p, const void* x, int B, int k, void* y, ui
     const int es = p->es, d = p->d, VEC = 16 / es;
     const int chunks = (d + 32 * VEC - 1) / (32 * VEC);
     // consumer warps / chunks per warp: least padding, CPW in {1, 2, 4}
-    static const int order[] = {8, 10, 12, 6, 7, 9, 11, 5, 4};
+    // tuning knob (read once): preferred number of consumer warps
+    static const int ncw_pref = getenv("POP_FUSED_WARPS") ? atoi(getenv("POP_FUSED_WARPS")) : 16;
+    const int order[] = {ncw_pref, 8, 10, 12, 16, 6, 7, 9, 11, 5, 4};
     int ncw = 0, CPW = 0, best = 1 << 30;
     for (int o : order) {
         int c = (chunks + o - 1) / o;

@@ -62,7 +62,8 @@ struct StreamParams {
     const float* wmax_cand;        // [2][n_cand] max |Wg[i][:]|, max |Wu[i][:]|
     double* margins;               // [n_cand] error bound of each approximate score
     const int32_t* idx_cand;
-    float* h;                      // [POP_MAX_BATCH][h_stride]
+    u64* h;                        // [POP_MAX_BATCH][h_stride] (float bits, epoch of the step that wrote them): a value
+                                   // carries its own validity, so publishing it needs no fence and no flag
     u64* keys;
     u32* keys32;                   // [n_cand] fp32 copies of the streamed scores (bit patterns)
     u64* uexact;                   // [n_cand] exact keys of the re-scored candidates (in job order)
@@ -70,7 +71,6 @@ struct StreamParams {
     float* y_acc;
     int32_t* sel_slots;
     u32* sync;
-    u32* flags;                    // [n_rt] epoch at which the unit's h was published
     uint8_t* mask_out;
     int32_t* sel_out;
     uint8_t* selflag;              // [n_cand] selection scratch: class / final flag of each candidate
@@ -185,6 +185,8 @@ __device__ __forceinline__ u32 split_bits(float v, int part) {
     return (u32)__bfloat16_as_ushort(r);
 }
 __device__ __forceinline__ u32 pack2(u32 lo, u32 hi) { return lo | (hi << 16); }
+
+__device__ __forceinline__ u64 h_word(float v, u32 epoch) { return (u64)__float_as_uint(v) | ((u64)epoch << 32); }
 
 #define POP_RAISE(code) do { ctrl->abort = 1; atomicExch(gerr, (u32)(code)); } while (0)
 
@@ -413,7 +415,7 @@ __device__ __noinline__ bool warp_selection(const StreamParams& P, Ctrl* ctrl, u
                             u += __ldcg(P.rpart + ((size_t)e * RPARTS + RPARTS / 2 + q) * POP_MAX_BATCH + bb);
                         }
                         const double hv = silu_f64(g) * u;
-                        P.h[(size_t)bb * P.h_stride + P.n_ret_pad + c] = (float)hv;
+                        P.h[(size_t)bb * P.h_stride + P.n_ret_pad + c] = h_word((float)hv, epoch);
                         energy = fma(hv, hv, energy);
                     }
                     P.uexact[e] = score_key(P.norm_cand[c] * sqrt(energy));
@@ -590,33 +592,43 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             ng = __shfl_sync(0xffffffffu, ng, 0);
             const int dslot = filled % ND;
             if (type == T_P2_RET) {
-                // wait for the h of the unit's channels: phase-1 units 2a .. 2(a+ng)-1
-                const int rt0 = 2 * a, rt1 = min(2 * (a + ng), P.n_rt);
-                if (lane < rt1 - rt0) {
-                    u32 sp = 0;
-                    while (ld_acquire_gpu(P.flags + rt0 + lane) != epoch) {
-                        if (ctrl->abort) { ok = false; break; }
-                        if (++sp > SPIN_LIMIT) { ctrl->abort = 1; atomicExch(gerr, (u32)ERR_FLAG); ok = false; break; }
-                        __nanosleep(64);
-                    }
-                }
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                for (int gi = 0; gi < ng; ++gi) {
+                // h of the unit's channels, as mma B fragments; a value not yet written this step (its
+                // epoch tag is old) is polled until the phase-1 unit that owns it has published it
+                for (int gi = 0; gi < ng && ok; ++gi) {
 #pragma unroll
                     for (int nb = 0; nb < NBLK; ++nb) {
                         const int n = g8 + 8 * nb, bb = n >> 1, part = n & 1;
                         u32 b0 = 0, b1 = 0;
                         if (bb < B) {
-                            const float* hp = P.h + (size_t)bb * P.h_stride + 16 * (a + gi);
-                            const float v0 = __ldcg(hp + 2 * t4), v1 = __ldcg(hp + 2 * t4 + 1);
-                            const float v2 = __ldcg(hp + 2 * t4 + 8), v3 = __ldcg(hp + 2 * t4 + 9);
-                            b0 = pack2(split_bits(v0, part), split_bits(v1, part));
-                            b1 = pack2(split_bits(v2, part), split_bits(v3, part));
+                            const u64* hp = P.h + (size_t)bb * P.h_stride + 16 * (a + gi);
+                            float v[4];
+                            u32 sp = 0;
+                            for (;;) {
+                                bool all = true;
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
+                                    if (16 * (a + gi) + kk < P.n_ret) {         // padding channels are zero
+                                        const u64 hw = __ldcg(hp + kk);
+                                        all = all && (u32)(hw >> 32) == epoch;
+                                        v[e] = __uint_as_float((u32)hw);
+                                    } else {
+                                        v[e] = 0.f;
+                                    }
+                                }
+                                if (all) break;
+                                if (ctrl->abort) { ok = false; break; }
+                                if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_FLAG); ok = false; break; }
+                                __nanosleep(64);
+                            }
+                            b0 = pack2(split_bits(v[0], part), split_bits(v[1], part));
+                            b1 = pack2(split_bits(v[2], part), split_bits(v[3], part));
                         }
                         hfrag[((dslot * MAXG + gi) * NBLK + nb) * 32 + lane] = make_uint2(b0, b1);
                     }
                 }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
             } else if (type == T_P2_CAND) {
                 if (lane == 0) {
                     u32 sp = 0;
@@ -642,7 +654,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     for (int e = 0; e < 4; ++e) {
                         const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
                         const int s = __shfl_sync(0xffffffffu, sc, kk);
-                        v[e] = (s >= 0 && bb < B) ? __ldcg(P.h + (size_t)bb * P.h_stride + P.n_ret_pad + s) : 0.f;
+                        v[e] = (s >= 0 && bb < B) ? __uint_as_float((u32)__ldcg(P.h + (size_t)bb * P.h_stride + P.n_ret_pad + s)) : 0.f;
                     }
                     hfrag[((dslot * MAXG + 0) * NBLK + nb) * 32 + lane] =
                         make_uint2(pack2(split_bits(v[0], part), split_bits(v[1], part)),
@@ -711,7 +723,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         us += pb[ww * PART_W + (ch + 8) * BCAP + nn];
                     }
                     const int slot = 8 * hdr.y + ch;
-                    if (nn < B && slot < P.n_ret) P.h[(size_t)nn * P.h_stride + slot] = silu_f32(gs) * us;
+                    if (nn < B && slot < P.n_ret) P.h[(size_t)nn * P.h_stride + slot] = h_word(silu_f32(gs) * us, epoch);
                 } else {
                     // Candidate unit: approximate score and a bound of its error.  The warps' partial sums are
                     // added in fp64 (exact for all practical purposes); each partial sum comes from S tensor-core
@@ -733,7 +745,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         dg *= P.cstep;
                         du *= P.cstep;
                         const double hv = silu_f64(gs) * us;
-                        P.h[(size_t)nn * P.h_stride + P.n_ret_pad + c2] = (float)hv;
+                        P.h[(size_t)nn * P.h_stride + P.n_ret_pad + c2] = h_word((float)hv, epoch);
                         // |silu'| <= 1.1
                         const double dh = 1.1 * dg * (fabs(us) + du) + fabs(silu_f64(gs)) * du + 1e-15 * fabs(hv);
                         e2 = hv * hv;
@@ -756,15 +768,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     }
                 }
             }
-            __threadfence();
+            if (is_cand) __threadfence();                    // keys and margins before the count below
             __syncwarp();
             int sel_now = 0;
             if (lane == 0) {
                 __threadfence_block();
                 ctrl->reduced = u + 1;
-                if (!is_cand) {
-                    st_release_gpu(P.flags + hdr.y, epoch);
-                } else {
+                if (is_cand) {
                     const u32 prev = atomicAdd(P.sync + SYNC_CAND_DONE, 1u);
                     sel_now = (prev == (u32)P.Uc - 1u) ? 1 : 0;
                     __threadfence();
@@ -1174,8 +1184,8 @@ int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void
     // before/after, any single product); taken twice over, and doubled again for safety.  The GPU tests check
     // the bound against the oracle's exact scores (observed error stays below 2 % of it).
     P.cstep = (double)(p->d / 16 / NCW) * 4.0 * (1.0 / 8388608.0);
-    P.norm_cand = p->norm_cand; P.idx_cand = p->idx_cand; P.h = p->h; P.keys = p->keys; P.y_acc = p->y_acc;
-    P.sel_slots = p->sel_slots; P.sync = p->sync; P.flags = p->flags; P.mask_out = mask_out; P.sel_out = sel_out;
+    P.norm_cand = p->norm_cand; P.idx_cand = p->idx_cand; P.h = reinterpret_cast<u64*>(p->h); P.keys = p->keys; P.y_acc = p->y_acc;
+    P.sel_slots = p->sel_slots; P.sync = p->sync; P.mask_out = mask_out; P.sel_out = sel_out;
     P.d = p->d; P.B = B; P.k = k; P.n_ret = p->n_ret; P.n_cand = p->n_cand; P.n_rt = p->n_rt; P.n_cg = p->n_cg;
     P.n_ret_pad = p->n_ret_pad; P.h_stride = p->h_stride;
     P.Uc = (p->n_cand + 7) / 8;

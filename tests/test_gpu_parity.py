@@ -235,3 +235,68 @@ def test_config2_full_size(r):
 def test_config5_full_size(batch):
     cfg = wl.config5(batch)
     run_case(cfg, steps=3)
+
+
+# ------------------------------------------------------------------ Mixtral-shaped MoE layer (composition of the two calls)
+def run_moe_case(cfg, n_experts, steps):
+    """One partition per expert from the prompt tokens routed to it, then per decode token the two routed
+    experts' decode steps combined with the renormalised router weights.  The router (softmax, top-2) and the
+    weighted sum are harness code in torch; every FFN step goes through the C ABI."""
+    m = wl.make_moe_workload(cfg, n_experts=n_experts, top_k=2, steps=steps)
+    dev = torch.device("cuda:0")
+    ratios = cfg.ratios.astuple()
+    ex_host = [tuple(np.asarray(a.values, dtype=np.float64) for a in (e.Wg, e.Wu, e.Wd)) for e in m.experts]
+    ref_parts = po.moe_prefill_partitions(m.X.values, ex_host, m.prompt_logits, ratios, 2)
+    # harness routing on the device
+    pl = torch.from_numpy(m.prompt_logits).to(dev)
+    top = torch.topk(torch.softmax(pl.double(), dim=-1), 2, dim=-1).indices
+    Xd = pr.to_dev(m.X)
+    parts = []
+    for e in range(n_experts):
+        tok = torch.nonzero((top == e).any(dim=1)).flatten()
+        assert np.array_equal(tok.cpu().numpy(), ref_parts[e]["tokens"])
+        Wg, Wu, Wd = (pr.to_dev(a) for a in (m.experts[e].Wg, m.experts[e].Wu, m.experts[e].Wd))
+        part = pop.prefill_partition(Xd[tok].contiguous(), Wg, Wu, Wd, ratios)
+        pr.check_regions(part, ref_parts[e])
+        parts.append(part)
+        del Wg, Wu, Wd
+    k = parts[0].n_cand // 2
+    worst = 0.0
+    for t in range(steps):
+        x = pr.to_dev(m.xs, index=t)
+        dl = torch.from_numpy(m.decode_logits[t]).to(dev).double()
+        p = torch.softmax(dl, dim=-1)
+        wts, ids = torch.topk(p, 2)
+        wts = wts / wts.sum()
+        o = po.moe_decode_step(m.xs.values[t, 0], ex_host, ref_parts, m.decode_logits[t], k, 2)
+        assert np.array_equal(np.sort(ids.cpu().numpy()), np.sort(o["experts"]))
+        y = torch.zeros(1, cfg.d, dtype=torch.float64, device=dev)
+        for j in range(2):
+            e = int(ids[j])
+            R, C, _ = parts[e].indices()
+            mask = torch.empty(parts[e].n_cand, dtype=torch.uint8, device=dev)
+            sel = torch.empty(k, dtype=torch.int32, device=dev)
+            ye = pop.decode_step(parts[e], x, k, mask_out=mask, sel_out=sel)
+            torch.cuda.synchronize()
+            parts[e].check()
+            oe = [po_e for po_e in o["per_expert"] if po_e[0] == e][0][2]
+            pr.check_selection(sel.cpu().numpy(), mask.cpu().numpy(), C, oe, k)
+            assert pr.rel_err(pr.host_values(ye), oe["y"]) <= pr.TOL[cfg.dtype]
+            y += float(wts[j]) * ye.double()
+        # The combined output: every expert output arrives rounded to bf16 (2^-9 of its own magnitude), which is
+        # an absolute error for the weighted sum where the experts cancel; it is judged normwise.
+        worst = max(worst, pr.normwise_err(y.cpu().numpy()[0], o["y"]))
+    assert worst <= 1e-2, f"MoE output error {worst:.3e}"
+    for part in parts:
+        part.destroy()
+
+
+def test_moe_small():
+    cfg = wl.FFNConfig("moe_small", d=2048, N=600, dtype=wl.BF16, prompt_tokens=48, decode_steps=3,
+                       ratios=wl.Ratios(0.5, 0.2, 0.3), seed=11)
+    run_moe_case(cfg, n_experts=4, steps=3)
+
+
+def test_config4_moe_full_size():
+    cfg = wl.config4_expert(0.2)
+    run_moe_case(cfg, n_experts=8, steps=2)
