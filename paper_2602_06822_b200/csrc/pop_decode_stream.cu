@@ -39,17 +39,18 @@ constexpr int NCW = 8;                     // consumer warps (16 / NCW must be a
 constexpr int NTC = NCW * 32;              // consumer threads
 constexpr int W_SCHED = NCW;               // scheduler warp
 constexpr int W_RED = NCW + 1;             // reducer warp
-constexpr int NTHREADS = NTC + 64;
+constexpr int W_SEL = NCW + 2;             // selection warp
+constexpr int NTHREADS = NTC + 96;
 constexpr int NPB_MAX = 4;                 // partial-sum buffers between the consumer warps and the reducer warp
 constexpr int ND = 8;                      // unit descriptors in flight per CTA
 constexpr int MAXG = 4;                    // copy groups per unit at most
 constexpr u32 SPIN_LIMIT = 1u << 22;       // polls (with a short sleep) before a wait gives up: seconds
-constexpr u32 BAR_SPIN_LIMIT = 1u << 20;   // mbarrier try_wait calls (each suspends for a while) before giving up
 constexpr int SLOT = 512;                  // bytes one warp copies per cp.async instruction
+constexpr int KPL = 48;                    // candidate keys per lane of a selection warp: n_cand <= 32 * KPL
 
 enum { T_P1_CAND = 0, T_P1_RET = 1, T_P2_RET = 2, T_P2_CAND = 3, T_END = 4 };
 enum { ERR_DESC = 11, ERR_PART_FULL = 12, ERR_FLAG = 13, ERR_SELECT_FLAG = 14, ERR_THROTTLE = 15, ERR_PART_FREE = 16,
-       ERR_REFINE = 17 };
+       ERR_REFINE = 17, ERR_CAND_DONE = 18 };
 
 struct StreamParams {
     const unsigned char* GUt;      // [n_rt][d/16][32][16 B]   retained gate/up fragments
@@ -60,20 +61,15 @@ struct StreamParams {
     __nv_bfloat16* y;
     const double* norm_cand;
     const float* wmax_cand;        // [2][n_cand] max |Wg[i][:]|, max |Wu[i][:]|
-    double* margins;               // [n_cand] error bound of each approximate score
     const int32_t* idx_cand;
     u64* h;                        // [POP_MAX_BATCH][h_stride] (float bits, epoch of the step that wrote them): a value
                                    // carries its own validity, so publishing it needs no fence and no flag
-    u64* keys;
-    u32* keys32;                   // [n_cand] fp32 copies of the streamed scores (bit patterns)
-    u64* uexact;                   // [n_cand] exact keys of the re-scored candidates (in job order)
+    uint2* km;                     // [n_cand] streamed score of each candidate and a bound of its error (two fp32 bit patterns)
     double* rpart;                 // [n_cand * RPARTS][POP_MAX_BATCH] partial dot products of the re-scoring jobs
     float* y_acc;
-    int32_t* sel_slots;
     u32* sync;
     uint8_t* mask_out;
     int32_t* sel_out;
-    uint8_t* selflag;              // [n_cand] selection scratch: class / final flag of each candidate
     int d, B, k, n_ret, n_cand, n_rt, n_cg, n_ret_pad, h_stride;
     int Uc, U1, n_cu, NG, NPB, p2_macro;
     double cstep;                  // error bound of one warp's partial dot product / the largest magnitude in it
@@ -87,16 +83,13 @@ struct Ctrl {
     volatile int filled;           // descriptors published by the scheduler
     volatile int abort;
     volatile int reduced;          // phase-1 units the reducer is done with
-    volatile int p1_total;         // phase-1 units this CTA consumed in all (-1 until known)
     int last;
     volatile int cons_m[NCW];
     volatile int cons_g[NCW];
     int cmt[NCW][8];               // consumer warps: commit index of each ring position
     float xmax[POP_MAX_BATCH];     // max |x[b][:]|
-    // exact re-scoring of uncertain candidates, shared out among the warps of the selecting CTA
-    volatile int rf_active;        // a job is posted
-    volatile int rf_n;             // entries of the job
-    int rf_next, rf_done;          // claimed / finished entries (atomics)
+    volatile int sel_final;        // this CTA's copy of the selection (rowmask) is final
+    u32 rowmask[KPL];              // bit l of word j: candidate 32 j + l is selected in this step
     u32 selsm[POP_SELECT_SMEM_WORDS(32)];
 };
 
@@ -174,9 +167,6 @@ __device__ __forceinline__ bool mbar_try_wait(u32 bar, u32 parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ void named_bar(int id, int nthreads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
-}
 
 // h as a bf16 pair: part 0 = nearest bf16, part 1 = nearest bf16 of the remainder.
 __device__ __forceinline__ u32 split_bits(float v, int part) {
@@ -190,129 +180,151 @@ __device__ __forceinline__ u64 h_word(float v, u32 epoch) { return (u64)__float_
 
 #define POP_RAISE(code) do { ctrl->abort = 1; atomicExch(gerr, (u32)(code)); } while (0)
 
+// Event timestamps for performance work: compiled in only with -DPOP_STREAM_TRACE (a build of its own);
+// slot `id` of the calling CTA gets the time at which its lane 0 passed the marker.
+#ifdef POP_STREAM_TRACE
+constexpr int TRACE_SLOTS = 32;
+__device__ unsigned long long g_trace[1024 * TRACE_SLOTS];
+__device__ __forceinline__ unsigned long long trace_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#define POP_TRACE(id) do { if (lane == 0) g_trace[cta * TRACE_SLOTS + (id)] = trace_now(); } while (0)
+#define POP_TRACE_VALUE(id, v) do { if (lane == 0) g_trace[cta * TRACE_SLOTS + (id)] = (unsigned long long)(v); } while (0)
+#else
+#define POP_TRACE(id) do { } while (0)
+#define POP_TRACE_VALUE(id, v) do { } while (0)
+#endif
+
 // ---------------------------------------------------------------------------------------------
-// Exact (fp64) re-scoring of uncertain candidates, as a job list posted in the control block.
-// Job e = (candidate ulist[e / RPARTS], part e % RPARTS): one part is a 1/(RPARTS/2) segment of the
-// candidate's gate row (parts < RPARTS/2) or up row; the warp that takes it returns the fp64 dot
-// products with x[b] over that segment in P.rpart[e][b].  Every warp of the CTA that calls this
-// takes jobs until none is left; all loads of a job are issued before the first is used (one
-// memory round trip per job and batch row).  A product of two bf16 values is exact in fp32; sums
-// in fp64.
+// Exact (fp64) re-scoring of an uncertain candidate, cut into RPARTS * B jobs: job (e, b) with
+// e = (uncertain candidate number e / RPARTS, part e % RPARTS); a part is a 1/(RPARTS/2) segment
+// of the candidate's gate row (parts < RPARTS/2) or up row.  The warp that runs it leaves the fp64
+// dot product with x[b] over that segment in P.rpart[e][b].  All loads of a job are issued before
+// the first is used (one memory round trip).  A product of two bf16 values is exact
+// in fp32; sums in fp64.
 // ---------------------------------------------------------------------------------------------
 constexpr int RPARTS = 4;
 constexpr int RVEC = 8;                    // 16-byte vectors per lane in flight for each of the two operands
 
-__device__ __noinline__ void refine_work(const StreamParams& P, Ctrl* ctrl, int lane) {
-    const int njobs = ctrl->rf_n;
-    const int d = P.d, B = P.B;
+__device__ __noinline__ void refine_job(const StreamParams& P, int c, int e, int bb, int lane) {
+    const int d = P.d;
     const int seg = d / (RPARTS / 2);                          // elements per segment
     const int segv = seg >> 3;                                 // 16-byte vectors per segment
-    for (;;) {
-        int e = 0;
-        if (lane == 0) e = atomicAdd(&ctrl->rf_next, 1);
-        e = __shfl_sync(0xffffffffu, e, 0);
-        if (e >= njobs) break;
-        const int c = __ldcg(P.sel_slots + e / RPARTS);
-        const int part = e % RPARTS;
-        const int which = part / (RPARTS / 2), sidx = part % (RPARTS / 2);
-        const uint4* wr = reinterpret_cast<const uint4*>(P.GUc + ((size_t)c * 2 + which) * (size_t)d * 2) + (size_t)sidx * segv;
+    const int part = e % RPARTS;
+    const int which = part / (RPARTS / 2), sidx = part % (RPARTS / 2);
+    const uint4* wr = reinterpret_cast<const uint4*>(P.GUc + ((size_t)c * 2 + which) * (size_t)d * 2) + (size_t)sidx * segv;
+    {
+        const uint4* xr = reinterpret_cast<const uint4*>(P.x + (size_t)bb * d) + (size_t)sidx * segv;
+        double a0 = 0.0, a1 = 0.0;
 #pragma unroll 1
-        for (int bb = 0; bb < B; ++bb) {
-            const uint4* xr = reinterpret_cast<const uint4*>(P.x + (size_t)bb * d) + (size_t)sidx * segv;
-            double a0 = 0.0, a1 = 0.0;
-#pragma unroll 1
-            for (int v0 = lane; v0 < segv; v0 += 32 * RVEC) {
-                uint4 rw[RVEC], rx[RVEC];
+        for (int v0 = lane; v0 < segv; v0 += 32 * RVEC) {
+            uint4 rw[RVEC], rx[RVEC];
 #pragma unroll
-                for (int t = 0; t < RVEC; ++t) {
-                    const bool in = v0 + 32 * t < segv;
-                    rw[t] = in ? __ldg(wr + v0 + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
-                    rx[t] = in ? __ldg(xr + v0 + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
-                }
+            for (int t = 0; t < RVEC; ++t) {
+                const bool in = v0 + 32 * t < segv;
+                rw[t] = in ? __ldg(wr + v0 + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
+                rx[t] = in ? __ldg(xr + v0 + 32 * t) : make_uint4(0u, 0u, 0u, 0u);
+            }
 #pragma unroll
-                for (int t = 0; t < RVEC; ++t) {
-                    float fw[8], fx[8];
-                    Elem<__nv_bfloat16>::unpack(rw[t], fw);
-                    Elem<__nv_bfloat16>::unpack(rx[t], fx);
+            for (int t = 0; t < RVEC; ++t) {
+                float fw[8], fx[8];
+                Elem<__nv_bfloat16>::unpack(rw[t], fw);
+                Elem<__nv_bfloat16>::unpack(rx[t], fx);
 #pragma unroll
-                    for (int j = 0; j < 8; j += 2) {
-                        a0 += (double)(fw[j] * fx[j]);
-                        a1 += (double)(fw[j + 1] * fx[j + 1]);
-                    }
+                for (int j = 0; j < 8; j += 2) {
+                    a0 += (double)(fw[j] * fx[j]);
+                    a1 += (double)(fw[j + 1] * fx[j + 1]);
                 }
             }
-            a0 += a1;
+        }
+        a0 += a1;
 #pragma unroll
-            for (int off = 16; off; off >>= 1) a0 += __shfl_xor_sync(0xffffffffu, a0, off);
-            if (lane == 0) P.rpart[(size_t)e * POP_MAX_BATCH + bb] = a0;
-        }
-        if (lane == 0) {
-            __threadfence();
-            atomicAdd(&ctrl->rf_done, 1);
-        }
+        for (int off = 16; off; off >>= 1) a0 += __shfl_xor_sync(0xffffffffu, a0, off);
+        if (lane == 0) P.rpart[(size_t)e * POP_MAX_BATCH + bb] = a0;
     }
 }
 
-constexpr int KPL = 48;                    // candidate keys per lane of the selecting warp: n_cand <= 32 * KPL
-
 // ---------------------------------------------------------------------------------------------
-// Top-k of the candidates by (score descending, channel id ascending), decided on EXACT scores,
-// by the reducer warp of the CTA that saw the step's last candidate unit.
+// Top-k of the candidates by (score descending, channel id ascending), decided on EXACT scores.
+// Every CTA's selection warp runs this same program on the same data and arrives at the same
+// mask, which it keeps in its own shared memory: nothing has to be published, and the warps that
+// stream weights never wait for another CTA's selection.  Only the fp64 re-scoring is shared out
+// (job e goes to CTA e mod G) and exchanged through global memory.
 //
-// The streamed scores a_i (fp32 copies in P.keys32) are approximate, each with a bound m_i of its
-// error (m = max m_i).  With tau = the k-th largest a_i:  a_i > tau + 2m  => i is in the exact
-// top-k (fewer than k candidates have a_j > tau, and every other one has an exact score below
-// i's); a_i < tau - 2m => i is not (the k candidates with a_j >= tau all beat it).  Only the
-// candidates in between are re-scored in fp64 from their plain rows (all warps of the CTA help)
-// and ranked exactly.
+// The streamed scores a_i (fp32, P.keys32) are approximate, each with a bound m_i of its error
+// (m = max m_i).  Let [tau_lo, tau_hi] be a bucket of key values that holds the k-th largest a_i.
+// a_i > tau_hi + 2m  => i is in the exact top-k (fewer than k candidates have a_j > tau_hi, and
+// every other one has an exact score below i's); a_i < tau_lo - 2m => i is not (the k candidates
+// with a_j >= tau_lo all beat it).  The candidates in between are re-scored in fp64 from their
+// plain rows and ranked exactly among themselves; the best k - |IN| of them complete the top-k.
 //
-// This code runs once per step in one warp, so it is written for few instruction bytes (rolled
-// loops over a lane-private array; lane owns candidates lane + 32 j) and fetches in batches of
-// independent loads: an instruction-cache miss or a memory round trip per element is what one
-// warp cannot hide.
+// One warp pays about 10 ns per dependent instruction, so the code is written for few
+// instructions (rolled loops; lane owns candidates lane + 32 j) and fetches in batches of
+// independent loads.
 // ---------------------------------------------------------------------------------------------
-__device__ __noinline__ bool warp_selection(const StreamParams& P, Ctrl* ctrl, unsigned char* smem, int lane, u32 epoch) {
+__device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, unsigned char* smem, int lane,
+                                            int cta, int G) {
     const int n = P.n_cand, k = P.k;
     const int rows = (n + 31) >> 5;
     u32* gerr = P.sync + SYNC_ERROR;
     u32* hist = ctrl->selsm;
     const u32 hist_u = smem_u32(hist);
-    int32_t* const ulist = P.sel_slots;
-    uint8_t* const selflag = P.selflag;
+    u32* const keys_sm = reinterpret_cast<u32*>(smem + P.off_sel);            // [KPL][32]
+    int* const ulist = reinterpret_cast<int*>(keys_sm + KPL * 32);             // [KPL * 32] uncertain candidates, ascending
+    u64* const uex = reinterpret_cast<u64*>(ulist + KPL * 32);                 // [KPL * 32] their exact keys
+    u32* const rowmask = ctrl->rowmask;
+    u32* const kr = keys_sm + lane;                                            // this lane's keys at stride 32
     const u32 lt = (1u << lane) - 1u;
-    u64 m_in = 0ull, m_un = 0ull;                          // bit j: candidate lane + 32 j is IN / uncertain
-    u32* const kr = reinterpret_cast<u32*>(smem + P.off_sel) + lane;      // [KPL][32]: this lane's keys at stride 32
-    if (k >= n) {
-        m_in = ~0ull;
-    } else if (k > 0) {
-        double mm = 0.0;
+
+    for (int j = lane; j < KPL; j += 32) {
+        const int left = n - 32 * j;
+        rowmask[j] = (k >= n && left > 0) ? (left >= 32 ? 0xffffffffu : ((1u << left) - 1u)) : 0u;
+    }
+    __syncwarp();
+    if (k > 0 && n > 0) {
+        // all candidate units of the step reduced (their h, keys and bounds are visible after the acquire)
+        bool ok = true;
+        if (lane == 0) {
+            u32 sp = 0;
+            while (ld_acquire_gpu(P.sync + SYNC_CAND_DONE) < (u32)P.Uc) {
+                if (ctrl->abort) { ok = false; break; }
+                if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_CAND_DONE); ok = false; break; }
+                __nanosleep(200);
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) return false;
+    }
+    POP_TRACE(1);
+    if (k > 0 && k < n) {
+        float mm = 0.f;
         u32 kor = 0u, kand = ~0u;
 #pragma unroll 1
-        for (int j0 = 0; j0 < rows; j0 += 16) {
-            u32 kk[16];
-            double mg[16];
+        for (int j0 = 0; j0 < rows; j0 += KPL / 2) {
+            uint2 kv[KPL / 2];
 #pragma unroll
-            for (int t = 0; t < 16; ++t) {
+            for (int t = 0; t < KPL / 2; ++t) {
                 const int i = lane + 32 * (j0 + t);
-                kk[t] = i < n ? __ldcg(P.keys32 + i) : 0u;
-                mg[t] = i < n ? __ldcg(P.margins + i) : 0.0;
+                kv[t] = i < n ? __ldcg(P.km + i) : make_uint2(0u, 0u);
             }
 #pragma unroll
-            for (int t = 0; t < 16; ++t) {
-                if (j0 + t < KPL) kr[32 * (j0 + t)] = kk[t];
-                if (lane + 32 * (j0 + t) < n) { kor |= kk[t]; kand &= kk[t]; }
-                mm = fmax(mm, mg[t]);
+            for (int t = 0; t < KPL / 2; ++t) {
+                kr[32 * (j0 + t)] = kv[t].x;
+                if (lane + 32 * (j0 + t) < n) { kor |= kv[t].x; kand &= kv[t].x; }
+                mm = fmaxf(mm, __uint_as_float(kv[t].y));
             }
         }
 #pragma unroll
         for (int off = 16; off; off >>= 1) {
-            mm = fmax(mm, __shfl_xor_sync(0xffffffffu, mm, off));
+            mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, off));
             kor |= __shfl_xor_sync(0xffffffffu, kor, off);
             kand &= __shfl_xor_sync(0xffffffffu, kand, off);
         }
         // The k-th largest key up to its low bits: radix passes of 8 bits, skipping digits that all keys share,
-        // at most two counted passes (one warp pays about 10 ns per instruction; the bucket of keys that
-        // agree with the k-th largest on the digits looked at is far narrower than the error bounds anyway).
+        // at most two counted passes (the bucket of keys that agree with the k-th largest on the digits looked
+        // at is far narrower than the error bounds anyway).
         const u32 differ = kor ^ kand;
         u32 prefix = 0, mask = 0;
         int rem = k, counted = 0;
@@ -325,7 +337,7 @@ __device__ __noinline__ bool warp_selection(const StreamParams& P, Ctrl* ctrl, u
             }
             for (int i = lane; i < 256; i += 32) hist[i] = 0;
             __syncwarp();
-#pragma unroll 1
+#pragma unroll 4
             for (int j = 0; j < rows; ++j) {
                 const u32 key = kr[32 * j];
                 if (lane + 32 * j < n && (key & mask) == prefix)
@@ -361,128 +373,110 @@ __device__ __noinline__ bool warp_selection(const StreamParams& P, Ctrl* ctrl, u
             __syncwarp();
         }
         // fewer than k keys lie above the bucket [prefix, prefix | ~mask], at least k at or above its lower end
-        const double tau_lo = (double)__uint_as_float(prefix);
-        const double tau_hi = (double)__uint_as_float(prefix | ~mask);
-        const double m2 = 2.0 * mm;
+        // thresholds as key bit patterns, rounded away from the bucket (keys are non-negative floats: they order
+        // like their bit patterns)
+        const double m2 = 2.0 * (double)mm;
+        const float t_in = __double2float_ru((double)__uint_as_float(prefix | ~mask) + m2);
+        const float t_out = __double2float_rd((double)__uint_as_float(prefix) - m2);
+        const u32 thr_in = __float_as_uint(t_in);
+        const u32 thr_out = t_out > 0.f ? __float_as_uint(t_out) : 0u;
         int nin = 0, nu = 0;
-#pragma unroll 1
+#pragma unroll 4
         for (int j = 0; j < rows; ++j) {
             const int i = lane + 32 * j;
-            int cls = 0;                                    // 0 out, 1 in, 2 uncertain
-            if (i < n) {
-                const double a = (double)__uint_as_float(kr[32 * j]);
-                cls = a > tau_hi + m2 ? 1 : (a < tau_lo - m2 ? 0 : 2);
-            }
-            const u32 bu = __ballot_sync(0xffffffffu, cls == 2);
-            if (cls == 2) { ulist[nu + __popc(bu & lt)] = i; m_un |= 1ull << j; }
-            if (cls == 1) m_in |= 1ull << j;
+            const u32 key = kr[32 * j];
+            const bool is_in = i < n && key > thr_in;
+            const bool is_un = i < n && !is_in && !(key < thr_out);
+            const u32 bu = __ballot_sync(0xffffffffu, is_un);
+            const u32 bi = __ballot_sync(0xffffffffu, is_in);
+            if (is_un) ulist[nu + __popc(bu & lt)] = i;
+            if (lane == 0) rowmask[j] = bi;
             nu += __popc(bu);
-            nin += __popc(__ballot_sync(0xffffffffu, cls == 1));
+            nin += __popc(bi);
         }
+        __syncwarp();
+        POP_TRACE(2);
+        POP_TRACE_VALUE(16, nu);
         if (nu > 0) {
-            __threadfence();
-            __syncwarp();
-            if (lane == 0) {
-                ctrl->rf_n = nu * RPARTS; ctrl->rf_next = 0; ctrl->rf_done = 0;
-                __threadfence_block();
-                ctrl->rf_active = 1;
+            const int njobs = nu * RPARTS * P.B;
+            int mine = 0;
+#pragma unroll 1
+            for (int jb = cta; jb < njobs; jb += G) {
+                const int e = jb / P.B;
+                refine_job(P, ulist[e / RPARTS], e, jb - e * P.B, lane);
+                ++mine;
             }
-            __syncwarp();
-            refine_work(P, ctrl, lane);
-            u32 sp = 0;
             bool ok = true;
-            while (*(volatile int*)&ctrl->rf_done < nu * RPARTS) {
-                if (ctrl->abort) { ok = false; break; }
-                if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_REFINE); ok = false; break; }
-                __nanosleep(50);
+            POP_TRACE(3);
+            if (lane == 0) {
+                if (mine) { __threadfence(); atomicAdd(P.sync + SYNC_RF_DONE, (u32)mine); }
+                u32 sp = 0;
+                while (ld_acquire_gpu(P.sync + SYNC_RF_DONE) < (u32)njobs) {
+                    if (ctrl->abort) { ok = false; break; }
+                    if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_REFINE); ok = false; break; }
+                    __nanosleep(100);
+                }
             }
-            __syncwarp();
-            if (lane == 0) ctrl->rf_active = 0;
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) return false;
-            __threadfence();
+            POP_TRACE(4);
             // exact scores from the parts (fixed order), lane = uncertain candidate
 #pragma unroll 1
-            for (int e0 = 0; e0 < nu; e0 += 32) {
-                const int e = e0 + lane;
-                if (e < nu) {
-                    const int c = __ldcg(ulist + e);
-                    double energy = 0.0;
-                    for (int bb = 0; bb < P.B; ++bb) {
-                        double g = 0.0, u = 0.0;
+            for (int e = lane; e < nu; e += 32) {
+                const int c = ulist[e];
+                double energy = 0.0;
+                for (int bb = 0; bb < P.B; ++bb) {
+                    double g = 0.0, u = 0.0;
 #pragma unroll
-                        for (int q = 0; q < RPARTS / 2; ++q) {
-                            g += __ldcg(P.rpart + ((size_t)e * RPARTS + q) * POP_MAX_BATCH + bb);
-                            u += __ldcg(P.rpart + ((size_t)e * RPARTS + RPARTS / 2 + q) * POP_MAX_BATCH + bb);
-                        }
-                        const double hv = silu_f64(g) * u;
-                        P.h[(size_t)bb * P.h_stride + P.n_ret_pad + c] = h_word((float)hv, epoch);
-                        energy = fma(hv, hv, energy);
+                    for (int q = 0; q < RPARTS / 2; ++q) {
+                        g += __ldcg(P.rpart + ((size_t)e * RPARTS + q) * POP_MAX_BATCH + bb);
+                        u += __ldcg(P.rpart + ((size_t)e * RPARTS + RPARTS / 2 + q) * POP_MAX_BATCH + bb);
                     }
-                    P.uexact[e] = score_key(P.norm_cand[c] * sqrt(energy));
+                    const double hv = silu_f64(g) * u;
+                    energy = fma(hv, hv, energy);
                 }
+                uex[e] = score_key(P.norm_cand[c] * sqrt(energy));
             }
-            __threadfence();
             __syncwarp();
-            // rank inside the uncertain set: the best k - |IN| of them complete the top-k
-            const u64* uexact = P.uexact;
+            // rank inside the uncertain set (ulist ascends, so position order is channel order)
             const int ku = k - nin;
 #pragma unroll 1
-            for (int e0 = 0; e0 < nu; e0 += 32) {
-                const int e = e0 + lane;
-                const u64 ke = e < nu ? __ldcg(uexact + e) : 0ull;
-                const int ce = e < nu ? __ldcg(ulist + e) : 0;
+            for (int e = lane; e < nu; e += 32) {
+                const u64 ke = uex[e];
                 int r = 0;
 #pragma unroll 1
-                for (int f0 = 0; f0 < nu; f0 += 32) {
-                    const int f = f0 + lane;
-                    const u64 kf0 = f < nu ? __ldcg(uexact + f) : 0ull;
-                    const int cf0 = f < nu ? __ldcg(ulist + f) : 0x7fffffff;
-                    const int cnt = min(32, nu - f0);
-#pragma unroll 1
-                    for (int t = 0; t < cnt; ++t) {
-                        const u64 kf = __shfl_sync(0xffffffffu, kf0, t);
-                        const int cf = __shfl_sync(0xffffffffu, cf0, t);
-                        r += (kf > ke || (kf == ke && cf < ce)) ? 1 : 0;
-                    }
+                for (int f = 0; f < nu; ++f) {
+                    const u64 kf = uex[f];
+                    r += (kf > ke || (kf == ke && f < e)) ? 1 : 0;
                 }
-                if (e < nu) selflag[ce] = r < ku ? 1 : 0;
+                if (r < ku) {
+                    const int ce = ulist[e];
+                    atomicOr(&rowmask[ce >> 5], 1u << (ce & 31));
+                }
             }
-            __threadfence();
             __syncwarp();
         }
     }
-    // ordered walk in batches of 8 rows: verdicts of the uncertain ones and channel ids first, then the stores
-    int32_t* const sel_slots = P.sel_slots;
-    int32_t* const sel_out = P.sel_out;
-    uint8_t* const mask_out = P.mask_out;
-    int base = 0;
+    __threadfence_block();
+    __syncwarp();
+    if (lane == 0) ctrl->sel_final = 1;
+    POP_TRACE(5);
+    // outputs: row j of the mask by CTA j mod G
 #pragma unroll 1
-    for (int j0 = 0; j0 < rows; j0 += 8) {
-        int chan[8];
-        int verdict[8];
+    for (int j = cta; j < rows; j += G) {
+        int base = 0;
+        for (int jj = lane; jj < j; jj += 32) base += __popc(rowmask[jj]);
 #pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const int j = j0 + t, i = lane + 32 * j;
-            chan[t] = (sel_out && i < n) ? __ldg(P.idx_cand + i) : 0;
-            verdict[t] = (i < n && ((m_un >> j) & 1ull)) ? (int)__ldcg(selflag + i) : 0;
-        }
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-            const int j = j0 + t, i = lane + 32 * j;
-            const bool sel = i < n && (((m_in >> j) & 1ull) || verdict[t]);
-            const u32 b = __ballot_sync(0xffffffffu, sel);
-            if (i < n && mask_out) mask_out[i] = sel ? 1 : 0;
-            if (sel) {
-                const int pos = base + __popc(b & lt);
-                sel_slots[pos] = i;
-                if (sel_out) sel_out[pos] = chan[t];
-            }
-            base += __popc(b);
+        for (int off = 16; off; off >>= 1) base += __shfl_xor_sync(0xffffffffu, base, off);
+        const u32 m = rowmask[j];
+        const int i = 32 * j + lane;
+        if (i < n) {
+            const bool sel = (m >> lane) & 1u;
+            if (P.mask_out) P.mask_out[i] = sel ? 1 : 0;
+            if (sel && P.sel_out) P.sel_out[base + __popc(m & lt)] = __ldg(P.idx_cand + i);
         }
     }
-    __threadfence();
-    __syncwarp();
-    if (lane == 0) st_release_gpu(P.sync + SYNC_SEL_READY, epoch);
+    POP_TRACE(6);
     return true;
 }
 
@@ -504,29 +498,33 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
     const int d = P.d, B = P.B, KT = d >> 4;
     Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem + P.off_ctrl);
     uint2* hfrag = reinterpret_cast<uint2*>(smem + P.off_hfrag);   // [ND][MAXG][NBLK][32]
-    int* rows = reinterpret_cast<int*>(smem + P.off_rows);          // [ND][16]
+    int* rows = reinterpret_cast<int*>(smem + P.off_rows);          // [ND][32]
     u32* gerr = P.sync + SYNC_ERROR;
     const int NPB = P.NPB;
     constexpr int PART_W = 2 * 16 * BCAP;   // floats a warp deposits per phase-1 unit: 16 rows x BCAP sums, then magnitudes
 
     if (tid == 0) {
-        ctrl->filled = 0; ctrl->abort = 0; ctrl->reduced = 0; ctrl->p1_total = -1; ctrl->last = 0;
-        ctrl->rf_active = 0; ctrl->rf_n = 0; ctrl->rf_next = 0; ctrl->rf_done = 0;
+        ctrl->filled = 0; ctrl->abort = 0; ctrl->reduced = 0; ctrl->last = 0;
+        ctrl->sel_final = 0;
         for (int b = 0; b < NPB_MAX; ++b) mbar_init(smem_u32(&ctrl->bar_full[b]), NCW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < NCW) { ctrl->cons_m[tid] = 0; ctrl->cons_g[tid] = 0; }
+#ifdef POP_STREAM_TRACE
+    if (tid < TRACE_SLOTS) g_trace[cta * TRACE_SLOTS + tid] = 0ull;
+#endif
     __syncthreads();
+    if (warp == 0) POP_TRACE(0);
 
     if (warp == W_SCHED) {
         // ================================================================= scheduler warp
         const u32 epoch = ld_acquire_gpu(P.sync + SYNC_EPOCH) + 1u;
         int stage = 0, nstatic = 0, qoff = 0, pend_lo = 0, pend_hi = 0, pend_q = 0;   // lane 0's state
+        bool sel_waited = false;
         u32 spec = 0;                      // result of a claim issued ahead of its use
         bool spec_valid = false;
         int filled = 0, sched_groups = 0;
         const int myq = cta & 3;
-        const int nq_groups = P.n_cg + P.n_cu;
         bool done = false, ok = true;
         while (!done && ok) {
             // room in the descriptor ring and in the look-ahead window?
@@ -550,12 +548,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             if (lane == 0) {
                 for (;;) {
                     if (pend_lo < pend_hi) {
-                        if (pend_lo < P.n_cg) {
-                            ng = min(pend_hi, P.n_cg) - pend_lo;
-                            type = T_P2_RET; a = pend_lo; b = pend_q; pend_lo += ng;
-                        } else {
-                            type = T_P2_CAND; a = pend_lo - P.n_cg; b = pend_q; ng = 1; pend_lo += 1;
-                        }
+                        ng = pend_hi - pend_lo;
+                        type = T_P2_RET; a = pend_lo; b = pend_q; pend_lo += ng;
                         break;
                     }
                     if (stage == 0) {
@@ -569,27 +563,59 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                             break;
                         }
                         stage = 1;
+                        POP_TRACE(7);
                     }
-                    if (qoff >= 4 || nq_groups == 0) { type = T_END; break; }
+                    if (stage == 1) {
+                        // retained groups of this CTA's quarter, then what is left of the other quarters
+                        if (qoff >= 4 || P.n_cg == 0) { stage = 2; qoff = 0; spec_valid = false; POP_TRACE(8); continue; }
+                        const int q = (myq + qoff) & 3;
+                        const u32 pu = spec_valid ? spec : atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)P.p2_macro);
+                        spec_valid = false;
+                        const int p = (int)pu;
+                        if (p < P.n_cg) {
+                            pend_lo = p; pend_hi = min(p + P.p2_macro, P.n_cg); pend_q = q;
+                            // the next claim on this quarter is issued now and used when this range is drained, so
+                            // that its latency overlaps the staging of this range
+                            spec = atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)P.p2_macro);
+                            spec_valid = true;
+                        } else {
+                            ++qoff;
+                        }
+                        continue;
+                    }
+                    // stage 2: selected candidate rows, one unit = one word of the mask (32 candidates), last of all
+                    if (qoff >= 4 || P.n_cu == 0) { type = T_END; break; }
+                    if (!sel_waited) {
+                        u32 sp = 0;
+                        while (!ctrl->sel_final) {
+                            if (ctrl->abort) { type = -1; break; }
+                            if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_SELECT_FLAG); type = -1; break; }
+                            __nanosleep(64);
+                        }
+                        if (type < 0) break;
+                        __threadfence_block();
+                        sel_waited = true;
+                        POP_TRACE(9);
+                    }
                     const int q = (myq + qoff) & 3;
-                    const u32 pu = spec_valid ? spec : atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)P.p2_macro);
+                    const u32 pu = spec_valid ? spec : atomicAdd(P.sync + SYNC_QC0 + 32 * q, 1u);
                     spec_valid = false;
-                    const int p = (int)pu;
-                    if (p < nq_groups) {
-                        pend_lo = p; pend_hi = min(p + P.p2_macro, nq_groups); pend_q = q;
-                        // the next claim on this quarter is issued now and used when this range is drained, so
-                        // that its latency overlaps the staging of this range
-                        spec = atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)P.p2_macro);
+                    if ((int)pu < P.n_cu) {
+                        spec = atomicAdd(P.sync + SYNC_QC0 + 32 * q, 1u);
                         spec_valid = true;
-                    } else {
-                        ++qoff;
+                        const int cnt = __popc(ctrl->rowmask[pu]);
+                        if (cnt == 0) continue;
+                        type = T_P2_CAND; a = (int)pu; b = q; ng = (cnt + 15) >> 4;
+                        break;
                     }
+                    ++qoff;
                 }
             }
             type = __shfl_sync(0xffffffffu, type, 0);
             a = __shfl_sync(0xffffffffu, a, 0);
             b = __shfl_sync(0xffffffffu, b, 0);
             ng = __shfl_sync(0xffffffffu, ng, 0);
+            if (type < 0) { ok = false; break; }
             const int dslot = filled % ND;
             if (type == T_P2_RET) {
                 // h of the unit's channels, as mma B fragments; a value not yet written this step (its
@@ -630,36 +656,44 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
             } else if (type == T_P2_CAND) {
-                if (lane == 0) {
-                    u32 sp = 0;
-                    while (ld_acquire_gpu(P.sync + SYNC_SEL_READY) != epoch) {
-                        if (ctrl->abort) { ok = false; break; }
-                        if (++sp > SPIN_LIMIT) { ctrl->abort = 1; atomicExch(gerr, (u32)ERR_SELECT_FLAG); ok = false; break; }
-                        __nanosleep(64);
+                // row list of the unit: the selected ones among candidates 32 a .. 32 a + 31, padded with -1
+                const u32 m = ctrl->rowmask[a];
+                int* rw = rows + dslot * 32;
+                rw[lane] = -1;
+                __syncwarp();
+                if ((m >> lane) & 1u) rw[__popc(m & ((1u << lane) - 1u))] = 32 * a + lane;
+                __syncwarp();
+                // their h as mma B fragments (written by the reducers of the candidate units, all of which the
+                // selection has waited for; the epoch tag is checked all the same)
+                for (int gi = 0; gi < ng && ok; ++gi) {
+#pragma unroll
+                    for (int nb = 0; nb < NBLK; ++nb) {
+                        const int n = g8 + 8 * nb, bb = n >> 1, part = n & 1;
+                        float v[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
+                            const int sc = rw[16 * gi + kk];
+                            v[e] = 0.f;
+                            if (sc >= 0 && bb < B) {
+                                const u64* hp = P.h + (size_t)bb * P.h_stride + P.n_ret_pad + sc;
+                                u32 sp = 0;
+                                for (;;) {
+                                    const u64 hw = __ldcg(hp);
+                                    if ((u32)(hw >> 32) == epoch) { v[e] = __uint_as_float((u32)hw); break; }
+                                    if (ctrl->abort) { ok = false; break; }
+                                    if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_FLAG); ok = false; break; }
+                                    __nanosleep(64);
+                                }
+                            }
+                        }
+                        hfrag[((dslot * MAXG + gi) * NBLK + nb) * 32 + lane] =
+                            make_uint2(pack2(split_bits(v[0], part), split_bits(v[1], part)),
+                                       pack2(split_bits(v[2], part), split_bits(v[3], part)));
                     }
                 }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                int sc = -1;                                   // candidate slot of row `lane` of the unit
-                if (lane < 16) {
-                    const int pos = 16 * a + lane;
-                    if (pos < P.k) sc = __ldcg(P.sel_slots + pos);
-                    rows[dslot * 16 + lane] = sc;
-                }
-#pragma unroll
-                for (int nb = 0; nb < NBLK; ++nb) {
-                    const int n = g8 + 8 * nb, bb = n >> 1, part = n & 1;
-                    float v[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
-                        const int s = __shfl_sync(0xffffffffu, sc, kk);
-                        v[e] = (s >= 0 && bb < B) ? __uint_as_float((u32)__ldcg(P.h + (size_t)bb * P.h_stride + P.n_ret_pad + s)) : 0.f;
-                    }
-                    hfrag[((dslot * MAXG + 0) * NBLK + nb) * 32 + lane] =
-                        make_uint2(pack2(split_bits(v[0], part), split_bits(v[1], part)),
-                                   pack2(split_bits(v[2], part), split_bits(v[3], part)));
-                }
             }
             if (lane == 0) ctrl->desc[dslot] = make_int4(type, a, b, ng);
             __syncwarp();
@@ -669,11 +703,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             if (lane == 0) ctrl->filled = filled;
             if (type == T_END) done = true;
         }
+        POP_TRACE(10);
     } else if (warp == W_RED) {
         // ================================================================= reducer warp
         // Turns the consumer warps' partial sums of a phase-1 unit into h (and, for a candidate unit,
-        // the approximate score keys with their error bounds), publishes the unit's flag, and runs
-        // the top-k once the step's last candidate unit is in.  The consumer warps never wait for it.
+        // the approximate score keys with their error bounds) and counts the candidate units done.
+        // The consumer warps never wait for it.
         const u32 epoch = ld_acquire_gpu(P.sync + SYNC_EPOCH) + 1u;
         // max |x[b][:]| for the error bounds of the candidate scores
         for (int bb = 0; bb < B; ++bb) {
@@ -693,22 +728,19 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         __syncwarp();
         const float* part = reinterpret_cast<const float*>(smem + P.off_part);   // [NPB][NCW][PART_W]
         int u = 0;                                   // phase-1 units reduced so far
+        const int p1_count = cta < P.U1 ? (P.U1 - cta + G - 1) / G : 0;   // phase 1 is dealt out statically
         bool ok = true;
-        while (ok) {
+        while (ok && u < p1_count) {
             const int buf = u % NPB;
             const u32 bar = smem_u32(&ctrl->bar_full[buf]);
             const u32 parity = (u32)(u / NPB) & 1u;
             u32 sp = 0;
-            bool got = false;
-            for (;;) {
-                if (mbar_try_wait(bar, parity)) { got = true; break; }
-                const int tot = ctrl->p1_total;
-                if (tot >= 0 && u >= tot) break;     // the CTA has no further phase-1 unit
+            while (!mbar_try_wait(bar, parity)) {
                 if (ctrl->abort) { ok = false; break; }
                 if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_PART_FULL); ok = false; break; }
                 __nanosleep(100);
             }
-            if (!got) break;
+            if (!ok) break;
             const int2 hdr = ctrl->part_hdr[buf];
             const float* pb = part + (size_t)buf * NCW * PART_W;
             const bool is_cand = hdr.x == T_P1_CAND;
@@ -761,29 +793,26 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         const double nc = P.norm_cand[c2];
                         const double key = nc * sqrt(e2);
                         const float kf = (float)key;
-                        P.keys[c2] = score_key(key);
-                        P.keys32[c2] = __float_as_uint(kf);
-                        // bound of |fp32 key - exact score|
-                        P.margins[c2] = nc * sqrt(d2) * (1.0 + 1e-9) + key * 1.3e-7;
+                        // bound of |fp32 key - exact score|, rounded up
+                        const float mf = __double2float_ru(nc * sqrt(d2) * (1.0 + 1e-9) + key * 1.3e-7);
+                        P.km[c2] = make_uint2(__float_as_uint(kf), __float_as_uint(mf));
                     }
                 }
             }
             if (is_cand) __threadfence();                    // keys and margins before the count below
             __syncwarp();
-            int sel_now = 0;
             if (lane == 0) {
                 __threadfence_block();
                 ctrl->reduced = u + 1;
-                if (is_cand) {
-                    const u32 prev = atomicAdd(P.sync + SYNC_CAND_DONE, 1u);
-                    sel_now = (prev == (u32)P.Uc - 1u) ? 1 : 0;
-                    __threadfence();
-                }
+                if (is_cand) atomicAdd(P.sync + SYNC_CAND_DONE, 1u);    // what the selection warps wait for
             }
-            sel_now = __shfl_sync(0xffffffffu, sel_now, 0);
-            if (sel_now && !warp_selection(P, ctrl, smem, lane, epoch)) ok = false;
+            if (is_cand) POP_TRACE(17);
             ++u;
         }
+        POP_TRACE(14);
+    } else if (warp == W_SEL) {
+        // ================================================================= selection warp
+        selection_main(P, ctrl, smem, lane, cta, G);
     } else {
         // ================================================================= consumer warps
         const int w = warp;
@@ -848,7 +877,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                 for (int j = 0; j < GSL; ++j) cp16(dst0 + j * SLOT + lane * 16, isrc + j * SLOT);
                 isrc += istep;
             } else {   // T_P2_CAND: 16 rows x CPR chunks, row r at chunk (r * CPR + c), swizzled when CPR == 8
-                const int* rw = rows + (im % ND) * 16;
+                const int* rw = rows + (im % ND) * 32 + ig * 16;
 #pragma unroll
                 for (int j = 0; j < GSL; ++j) {
                     const int f = j * 32 + lane, r = f / CPR, c = f - r * CPR;
@@ -931,15 +960,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             }
         };
 
-        // Help with a posted re-scoring job (the selection runs in this CTA's reducer warp).
-        auto help_refine = [&]() {
-            if (ctrl->rf_active) { __threadfence_block(); refine_work(P, ctrl, lane); }
-        };
         // The partial-sum buffer of phase-1 unit number p1seq must have been released by the reducer.
         auto part_buffer_free = [&]() -> bool {
             u32 sp = 0;
             while (ctrl->reduced < p1seq - NPB + 1) {
-                help_refine();                       // the reducer may be waiting for this very help
                 if (ctrl->abort) return false;
                 if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_PART_FREE); return false; }
                 __nanosleep(20);
@@ -948,7 +972,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         };
 
         while (ok) {
-            help_refine();
             // descriptor of the unit to consume
             {
                 u32 sp = 0;
@@ -964,6 +987,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             const int dslot = cm % ND;
             if (cd.x == T_END) break;
             const bool is_p1 = cd.x <= T_P1_RET, is_cand = cd.x == T_P1_CAND;
+#ifdef POP_STREAM_TRACE
+            if (w == 0 && cd.x == T_P2_RET && cq < 0) POP_TRACE(11);
+            if (w == 0 && cd.x == T_P2_CAND && !g_trace[cta * TRACE_SLOTS + 12]) POP_TRACE(12);
+#endif
 
             // ---- unit prologue
             float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
@@ -1024,7 +1051,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     __syncwarp();                       // lanes read what other lanes copied
                     uint2 hb[NBLK];
 #pragma unroll
-                    for (int nb = 0; nb < NBLK; ++nb) hb[nb] = lds64(hf0 + (u32)(nb * 32) * 8u);
+                    for (int nb = 0; nb < NBLK; ++nb) hb[nb] = lds64(hf0 + (u32)((gi * NBLK + nb) * 32) * 8u);
                     const int mi = lane >> 3;
                     const int r = ((mi >> 1) << 3) + (lane & 7);
 #pragma unroll
@@ -1039,7 +1066,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                 }
                 ++n;
                 if (lane == 0) ctrl->cons_g[w] = n;
-                help_refine();
             }
             if (!ok) break;
 
@@ -1073,7 +1099,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             ++cm;
             if (lane == 0) ctrl->cons_m[w] = cm;
         }
-        if (tid == 0) { __threadfence_block(); ctrl->p1_total = p1seq; }
+        if (w == 0) POP_TRACE(13);
         cp_wait<0>();
         if (ok && !ctrl->abort && cq >= 0) flush(cq);
         __threadfence();
@@ -1081,6 +1107,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
 
     // ========================================================================= finish
     __syncthreads();
+    if (warp == 0) POP_TRACE(15);
     if (tid == 0) {
         const u32 ticket = atomicAdd(P.sync + SYNC_TICKET, 1u);
         __threadfence();
@@ -1089,10 +1116,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
     __syncthreads();
     if (ctrl->last) {
         // every CTA has added its partial sums: cast, clear the accumulator, re-arm the counters
-        for (int i = tid; i < B * d; i += NTHREADS) {
-            const float v = __ldcg(P.y_acc + i);
-            P.y[i] = __float2bfloat16_rn(v);
-            P.y_acc[i] = 0.f;
+        float4* ya = reinterpret_cast<float4*>(P.y_acc);
+        uint2* yo = reinterpret_cast<uint2*>(P.y);
+#pragma unroll 4
+        for (int i = tid; i < (B * d) >> 2; i += NTHREADS) {
+            const float4 v = __ldcg(ya + i);
+            yo[i] = make_uint2(pack2(split_bits(v.x, 0), split_bits(v.y, 0)), pack2(split_bits(v.z, 0), split_bits(v.w, 0)));
+            ya[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         __syncthreads();
         if (tid == 0) {
@@ -1100,11 +1130,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             P.sync[SYNC_P1] = 0;
             P.sync[SYNC_CAND_DONE] = 0;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) P.sync[SYNC_Q0 + 32 * q] = 0;
+            for (int q = 0; q < 4; ++q) { P.sync[SYNC_Q0 + 32 * q] = 0; P.sync[SYNC_QC0 + 32 * q] = 0; }
+            P.sync[SYNC_RF_DONE] = 0;
             const u32 epoch = P.sync[SYNC_EPOCH] + 1u;
             __threadfence();
             st_release_gpu(P.sync + SYNC_EPOCH, epoch);
         }
+        if (warp == 0) POP_TRACE(18);
     }
 }
 
@@ -1116,10 +1148,10 @@ int launch_stream(StreamParams& P, const pop_partition* p, cudaStream_t st) {
     // shared-memory layout: [ring][part][hfrag][rows][ystage][ctrl]
     const int GSL = GS * (16 / NCW);
     const int NPB = NBLK == 1 ? 3 : 2;
-    const int sel_bytes = KPL * 32 * 4;                        // the selecting warp's copy of the candidate keys
+    const int sel_bytes = KPL * 32 * (4 + 4 + 8);              // selection warp: candidate keys, uncertain list, exact keys
     const int part_bytes = NPB * NCW * 2 * 16 * (4 * NBLK) * 4;
     const int hfrag_bytes = ND * MAXG * NBLK * 32 * 8;
-    const int rows_bytes = ND * 16 * 4;
+    const int rows_bytes = ND * 32 * 4;
     const int ystage_bytes = NCW * GSL * 16 * 4;
     const int fixed = align_up(part_bytes, 128) + align_up(hfrag_bytes, 128) + align_up(rows_bytes, 128) +
                       align_up(ystage_bytes, 128) + align_up(sel_bytes, 128) + align_up((int)sizeof(Ctrl), 128);
@@ -1127,7 +1159,7 @@ int launch_stream(StreamParams& P, const pop_partition* p, cudaStream_t st) {
     int NG = (p->max_smem_optin - 1024 - fixed) / group_bytes;
     if (NG > 8) NG = 8;
     // tuning knob (read once): cap of the ring depth in copy groups
-    static const int ng_cap = getenv("POP_RING_GROUPS") ? atoi(getenv("POP_RING_GROUPS")) : 8;
+    static const int ng_cap = getenv("POP_RING_GROUPS") ? atoi(getenv("POP_RING_GROUPS")) : 3;
     if (NG > ng_cap) NG = ng_cap;
     if (NG < 3) return POP_ERR_UNSUPPORTED;
     P.NG = NG;
@@ -1152,12 +1184,28 @@ int launch_stream(StreamParams& P, const pop_partition* p, cudaStream_t st) {
         cfg_dev = dev; cfg_smem = smem_bytes; cfg_ok = per_sm >= 1;
     }
     if (!cfg_ok) return POP_ERR_UNSUPPORTED;
-    kern<<<p->sm_count, NTHREADS, smem_bytes, st>>>(P);
+    // CTAs wait on one another's results: a cooperative launch makes the driver place them all at once or refuse
+    static const int coop_env = getenv("POP_STREAM_COOP") ? atoi(getenv("POP_STREAM_COOP")) : 1;
+    if (p->coop && coop_env) {
+        void* args[] = {(void*)&P};
+        POP_CUDA(cudaLaunchCooperativeKernel((const void*)kern, dim3(p->sm_count), dim3(NTHREADS), args, smem_bytes, st));
+    } else {
+        kern<<<p->sm_count, NTHREADS, smem_bytes, st>>>(P);
+    }
     POP_LAUNCHED();
     return POP_OK;
 }
 
 }  // namespace
+
+#ifdef POP_STREAM_TRACE
+// Copies the event timestamps of the last launch to the host (trace builds only): [ctas][32].
+extern "C" int pop_debug_stream_trace(unsigned long long* h_out, int ctas) {
+    POP_CUDA(cudaDeviceSynchronize());
+    POP_CUDA(cudaMemcpyFromSymbol(h_out, g_trace, sizeof(unsigned long long) * 32 * (size_t)ctas));
+    return POP_OK;
+}
+#endif
 
 bool pop_stream_layout_supported(int d, pop_dtype_t dt) {
     if (dt != POP_BF16 || d % 1024 != 0) return false;
@@ -1177,25 +1225,21 @@ int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void
     P.WdTt = (const unsigned char*)p->WdT;
     P.WdTc = P.WdTt + (size_t)p->n_ret_pad * row;
     P.x = (const __nv_bfloat16*)x; P.y = (__nv_bfloat16*)y;
-    P.wmax_cand = p->wnorm_cand; P.margins = p->margins; P.selflag = p->selflag; P.keys32 = p->keys32; P.uexact = p->uexact; P.rpart = p->rpart;
+    P.wmax_cand = p->wnorm_cand; P.km = reinterpret_cast<uint2*>(p->keys); P.rpart = p->rpart;
     // Error model of a warp's partial dot product (d/16/NCW mma steps, each adding 16 exact bf16 x bf16 products to
     // an fp32 accumulator): the tensor core adds the 17 terms in a wider fixed-point format aligned to the largest
     // of them and rounds once, so one step errs by at most 2^-23 of the largest magnitude involved (accumulator
     // before/after, any single product); taken twice over, and doubled again for safety.  The GPU tests check
     // the bound against the oracle's exact scores (observed error stays below 2 % of it).
     P.cstep = (double)(p->d / 16 / NCW) * 4.0 * (1.0 / 8388608.0);
-    P.norm_cand = p->norm_cand; P.idx_cand = p->idx_cand; P.h = reinterpret_cast<u64*>(p->h); P.keys = p->keys; P.y_acc = p->y_acc;
-    P.sel_slots = p->sel_slots; P.sync = p->sync; P.mask_out = mask_out; P.sel_out = sel_out;
+    P.norm_cand = p->norm_cand; P.idx_cand = p->idx_cand; P.h = reinterpret_cast<u64*>(p->h); P.y_acc = p->y_acc;
+    P.sync = p->sync; P.mask_out = mask_out; P.sel_out = sel_out;
     P.d = p->d; P.B = B; P.k = k; P.n_ret = p->n_ret; P.n_cand = p->n_cand; P.n_rt = p->n_rt; P.n_cg = p->n_cg;
     P.n_ret_pad = p->n_ret_pad; P.h_stride = p->h_stride;
     P.Uc = (p->n_cand + 7) / 8;
     P.U1 = P.Uc + p->n_rt;
-    P.n_cu = (k + 15) / 16;
+    P.n_cu = k > 0 ? (p->n_cand + 31) / 32 : 0;
     P.p2_macro = p2_macro_env < 1 ? 1 : (p2_macro_env > MAXG ? MAXG : p2_macro_env);
-    if (P.Uc == 0) {
-        // no candidate unit will ever run the selection: nothing to select, publish that at once
-        // (mask_out has no entries, k == 0)
-    }
     const int gs = p->d / 1024;
     const int nblk = B <= 4 ? 1 : 2;
 #define POP_CASE(G_, N_) if (gs == G_ && nblk == N_) return launch_stream<G_, N_>(P, p, st);
