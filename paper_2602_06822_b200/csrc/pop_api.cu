@@ -89,11 +89,12 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device);
     cudaDeviceGetAttribute(&p->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
     const size_t row = (size_t)d * p->es;
-    // POP_DECODE_IMPL (read at every partition creation) picks the decode kernel family: "stream" = tiled layout +
-    // the dataflow kernel of pop_decode_stream.cu for the bf16 shapes it takes (its one-warp selection holds up to
-    // 1536 candidate keys); anything else = row layout + the fused / simple kernels.
+    // POP_DECODE_IMPL (read at every partition creation) picks the decode kernel family.  Unset or "stream": tiled
+    // layout + the dataflow kernel of pop_decode_stream.cu for the bf16 shapes it takes (its one-warp selection holds
+    // up to 1536 candidate keys), row layout + the fused / simple kernels for every other shape; "fused" or "simple":
+    // row layout and those kernels for all shapes.
     const char* impl = getenv("POP_DECODE_IMPL");
-    const bool want_stream = impl && !strcmp(impl, "stream");
+    const bool want_stream = !impl || !*impl || !strcmp(impl, "stream");
     p->layout = (want_stream && pop_stream_layout_supported(d, dt) && n_cand <= 1536) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
     p->n_rt = (n_ret + 7) / 8;
     p->n_cg = (n_ret + 15) / 16;

@@ -510,6 +510,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < NCW) { ctrl->cons_m[tid] = 0; ctrl->cons_g[tid] = 0; }
+    // When launched with programmatic stream serialization the CTA may have started while the previous kernel of
+    // the stream was still running: nothing of global memory is touched before that kernel is complete.  The next
+    // kernel may be placed from now on (it takes an SM only once a CTA of this one has left it).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 #ifdef POP_STREAM_TRACE
     if (tid < TRACE_SLOTS) g_trace[cta * TRACE_SLOTS + tid] = 0ull;
 #endif
@@ -521,6 +526,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         const u32 epoch = ld_acquire_gpu(P.sync + SYNC_EPOCH) + 1u;
         int stage = 0, nstatic = 0, qoff = 0, pend_lo = 0, pend_hi = 0, pend_q = 0;   // lane 0's state
         bool sel_waited = false;
+        int spec_amt = 0, cand_exh = 0;     // cand_exh bit q: the candidate units of quarter q are all claimed
+        const int cpq = (G + 3) >> 2;      // CTAs that start on the same quarter
         u32 spec = 0;                      // result of a claim issued ahead of its use
         bool spec_valid = false;
         int filled = 0, sched_groups = 0;
@@ -568,15 +575,37 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     if (stage == 1) {
                         // retained groups of this CTA's quarter, then what is left of the other quarters
                         if (qoff >= 4 || P.n_cg == 0) { stage = 2; qoff = 0; spec_valid = false; POP_TRACE(8); continue; }
+                        // Once the selection is final, the selected candidate rows of the quarter this CTA works on
+                        // come first: they are small gathered units, better placed where retained groups follow
+                        // than at the very end.
+                        {
+                            const int q = (myq + qoff) & 3;
+                            if (P.n_cu > 0 && !((cand_exh >> q) & 1) && ctrl->sel_final) {
+                                __threadfence_block();
+                                const int pc = (int)atomicAdd(P.sync + SYNC_QC0 + 32 * q, 1u);
+                                if (pc < P.n_cu) {
+                                    const int cnt = __popc(ctrl->rowmask[pc]);
+                                    if (cnt == 0) continue;
+                                    type = T_P2_CAND; a = pc; b = q; ng = (cnt + 15) >> 4;
+                                    break;
+                                }
+                                cand_exh |= 1 << q;
+                            }
+                        }
+                        // Claims shrink towards the end of a quarter (large ones keep the claim rate low, small ones
+                        // even out the finish): up to p2_macro groups while plenty are left, then 2, then 1.
                         const int q = (myq + qoff) & 3;
-                        const u32 pu = spec_valid ? spec : atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)P.p2_macro);
+                        const int amt0 = spec_valid ? spec_amt : P.p2_macro;
+                        const u32 pu = spec_valid ? spec : atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)amt0);
                         spec_valid = false;
                         const int p = (int)pu;
                         if (p < P.n_cg) {
-                            pend_lo = p; pend_hi = min(p + P.p2_macro, P.n_cg); pend_q = q;
+                            pend_lo = p; pend_hi = min(p + amt0, P.n_cg); pend_q = q;
                             // the next claim on this quarter is issued now and used when this range is drained, so
                             // that its latency overlaps the staging of this range
-                            spec = atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)P.p2_macro);
+                            const int left = P.n_cg - pend_hi;
+                            spec_amt = left >= 6 * cpq ? P.p2_macro : (left >= 2 * cpq ? min(2, P.p2_macro) : 1);
+                            spec = atomicAdd(P.sync + SYNC_Q0 + 32 * q, (u32)spec_amt);
                             spec_valid = true;
                         } else {
                             ++qoff;
@@ -598,6 +627,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         POP_TRACE(9);
                     }
                     const int q = (myq + qoff) & 3;
+                    if ((cand_exh >> q) & 1) { ++qoff; continue; }
                     const u32 pu = spec_valid ? spec : atomicAdd(P.sync + SYNC_QC0 + 32 * q, 1u);
                     spec_valid = false;
                     if ((int)pu < P.n_cu) {
@@ -1185,8 +1215,25 @@ int launch_stream(StreamParams& P, const pop_partition* p, cudaStream_t st) {
     }
     if (!cfg_ok) return POP_ERR_UNSUPPORTED;
     // CTAs wait on one another's results: a cooperative launch makes the driver place them all at once or refuse
-    static const int coop_env = getenv("POP_STREAM_COOP") ? atoi(getenv("POP_STREAM_COOP")) : 1;
-    if (p->coop && coop_env) {
+    // POP_STREAM_LAUNCH (read once): "pdl" (default) = plain launch with programmatic stream serialization, which lets
+    // this kernel's CTAs take the SMs the previous kernel of the stream leaves, up to their griddepcontrol.wait, and
+    // so hides the launch latency between the steps of a decode loop; "coop" = cooperative launch, which makes the
+    // driver place all CTAs at once even when other streams keep SMs busy, at the price of that latency; "plain".
+    // In the first and last mode a CTA that could not be placed alongside the others makes the bounded waits of
+    // the others expire (status POP_ERR_TIMEOUT from pop_partition_check), not hang.
+    static const char* launch_env = getenv("POP_STREAM_LAUNCH");
+    static const int pdl_env = !launch_env || !*launch_env || !strcmp(launch_env, "pdl");
+    static const int coop_env = launch_env && !strcmp(launch_env, "coop");
+    if (pdl_env) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3(p->sm_count); cfg.blockDim = dim3(NTHREADS); cfg.dynamicSmemBytes = smem_bytes; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        POP_CUDA(cudaLaunchKernelEx(&cfg, kern, P));
+    } else if (p->coop && coop_env) {
         void* args[] = {(void*)&P};
         POP_CUDA(cudaLaunchCooperativeKernel((const void*)kern, dim3(p->sm_count), dim3(NTHREADS), args, smem_bytes, st));
     } else {
