@@ -320,6 +320,8 @@ def run_pop(args):
             "e2e": {"value": e2e_value, "unit": "layer-steps/s",
                     "h2d_bytes_per_step": int(X_host.numel() * es + tokens * B * d * es),
                     "d2h_bytes_per_step": int(tokens * B * d * es),
+                    "prefill_ms_per_step": e2e["prefill_ms"] / e2e_steps,
+                    "decode_ms_per_step": e2e["decode_ms"] / e2e_steps,
                     "note": "prompt copied from pinned host memory before prefill; per token x copied in, last layer's y "
                             "copied out and the stream synchronised"},
             "gpu_launches": int(res["launches"]),

@@ -72,7 +72,7 @@ static void partition_free(pop_partition* p) {
     if (!p) return;
     cudaFree(p->GU); cudaFree(p->WdT); cudaFree(p->idx_ret); cudaFree(p->idx_cand); cudaFree(p->idx_pruned);
     cudaFree(p->scores); cudaFree(p->norm_cand); cudaFree(p->h); cudaFree(p->keys); cudaFree(p->y_acc);
-    cudaFree(p->sel_slots); cudaFree(p->sync); cudaFree(p->flags); cudaFree(p->wnorm_cand); cudaFree(p->margins); cudaFree(p->selflag); cudaFree(p->keys32); cudaFree(p->uexact); cudaFree(p->rpart);
+    cudaFree(p->sel_slots); cudaFree(p->sync); cudaFree(p->wnorm_cand); cudaFree(p->rpart);
     free(p);
 }
 
@@ -120,18 +120,12 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     TRY(dev_alloc(&p->y_acc, sizeof(float) * (size_t)POP_MAX_BATCH * d));
     TRY(dev_alloc(&p->sel_slots, sizeof(int32_t) * (size_t)n_cand));
     TRY(dev_alloc(&p->sync, sizeof(u32) * SYNC_WORDS));
-    TRY(dev_alloc(&p->flags, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1)));
     TRY(dev_alloc(&p->wnorm_cand, sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1)));
-    TRY(dev_alloc(&p->margins, sizeof(double) * (size_t)(n_cand > 0 ? n_cand : 1)));
-    TRY(dev_alloc(&p->selflag, (size_t)(n_cand > 0 ? n_cand : 1)));
-    TRY(dev_alloc(&p->keys32, sizeof(u32) * (size_t)(n_cand > 0 ? n_cand : 1)));
-    TRY(dev_alloc(&p->uexact, sizeof(u64) * (size_t)(n_cand > 0 ? n_cand : 1)));
     TRY(dev_alloc(&p->rpart, sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1)));
 #undef TRY
     e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->scores, 0, sizeof(double) * (size_t)N, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p->flags, 0, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1), st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1), st);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free(p); return POP_ERR_CUDA; }
     *out = p;
@@ -277,7 +271,6 @@ extern "C" int pop_partition_check(pop_partition_t* p) {
         // leave the partition usable: clear counters and the accumulator
         POP_CUDA(cudaMemset(p->sync, 0, sizeof(u32) * SYNC_WORDS));
         POP_CUDA(cudaMemset(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * p->d));
-        POP_CUDA(cudaMemset(p->flags, 0, sizeof(u32) * (size_t)(p->n_rt > 0 ? p->n_rt : 1)));
         POP_CUDA(cudaMemset(p->h, 0, 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1)));
         return POP_ERR_TIMEOUT;
     }

@@ -55,19 +55,16 @@ struct pop_partition {
     double* scores;               // [N] prefill I_i
     double* norm_cand;            // [n_cand] ||Wd[:, i]||_2 of the candidate channels
     float* wnorm_cand;            // [2][n_cand] max |Wg[i][:]|, max |Wu[i][:]| of the candidate channels
-    double* margins;              // [n_cand] decode scratch: error bound of each approximate candidate score
-    uint8_t* selflag;             // [n_cand] decode scratch of the selection
-    u32* keys32;                  // [n_cand] decode scratch: fp32 copies of the streamed candidate scores
-    u64* uexact;                  // [n_cand] decode scratch: exact keys of re-scored candidates
     double* rpart;                // [4 n_cand][POP_MAX_BATCH] decode scratch: partial dot products of re-scoring jobs
 
     // decode scratch (no allocation at decode time)
-    float* h;                     // [POP_MAX_BATCH][n_rc] intermediate activations of this step
-    u64* keys;                    // [n_cand] candidate scores as ordered 64-bit keys
+    float* h;                     // intermediate activations of this step: [POP_MAX_BATCH][n_rc] floats (row layout);
+                                  // tiled layout: [POP_MAX_BATCH][h_stride] 8-byte words (float bits, epoch of the step)
+    u64* keys;                    // [n_cand] candidate scores as ordered 64-bit keys (row layout); tiled layout:
+                                  // (streamed fp32 score, bound of its error) as two 32-bit patterns
     float* y_acc;                 // [POP_MAX_BATCH][d] fp32 accumulator, zero between steps
     int32_t* sel_slots;           // [n_cand] selected candidate slots (ascending), this step
     u32* sync;                    // [SYNC_WORDS] counters / flags, see pop_decode*.cu
-    u32* flags;                   // [n_rt] tiled layout: epoch at which a phase-1 unit published its h
     int sm_count;
     int coop;                     // device supports cooperative launch
     int max_smem_optin;
@@ -75,7 +72,7 @@ struct pop_partition {
 
 // sync[] word assignment (contended counters sit on separate 128-byte lines)
 enum { SYNC_BARRIER = 0, SYNC_TICKET = 1, SYNC_ERROR = 2, SYNC_WORK = 3,
-       SYNC_EPOCH = 32, SYNC_P1 = 64, SYNC_CAND_DONE = 96,
+       SYNC_EPOCH = 32, SYNC_CAND_DONE = 96,
        SYNC_Q0 = 128 /* + 32 q, q = 0..3 */, SYNC_QC0 = 256 /* + 32 q */, SYNC_RF_DONE = 384,
        SYNC_WORDS = 416 };
 

@@ -1,32 +1,43 @@
 // Decode step of POP (Sec. 3.3 "Decoding Stage", Sec. 3.4) for bf16 partitions in the tiled
-// layout: ONE persistent kernel without any grid-wide barrier.  The step is cut into work units
-// that CTAs claim from device-side counters; a unit that depends on another unit's result waits
-// for that unit's flag only, so fast SMs run ahead instead of idling at a barrier.
+// layout: ONE persistent kernel without any grid-wide barrier.  The step is cut into work units;
+// a unit that depends on another unit's result waits for that result only, so fast SMs run ahead
+// instead of idling at a barrier.
 //
-//   phase-1 unit, Candidate   8 candidate channels: gate/up rows in fp64 (their scores decide the
-//                             mask), h = silu(g) * u, score keys.  These units come first in the
-//                             queue; the CTA that completes the last of them runs the exact
-//                             radix top-k at once, while everybody else streams Retained rows.
-//   phase-1 unit, Retained    8 retained channels: 16 rows (8 gate + 8 up) x d on the tensor
+//   phase-1 unit, Candidate   8 candidate channels: 16 rows (8 gate + 8 up) x d on the tensor
 //                             cores (mma.m16n8k16, bf16 x bf16 -> fp32; the batch is the n dimension),
-//                             h published with a per-unit ready flag.
-//   phase-2 unit, Retained    16 retained channels x one quarter of the d outputs, again as
-//                             m16n8k16 tiles; h enters as a bf16 (high, low) pair in two columns
-//                             of the n dimension, so that y keeps fp32 accuracy.
-//   phase-2 unit, Candidate   16 selected candidate rows x one quarter of d (only selected rows
-//                             are read), gathered by row id, transposed by ldmatrix.
+//                             together with the largest magnitudes met, from which a bound of the
+//                             error of the score follows.  These units come first.
+//   phase-1 unit, Retained    8 retained channels, the same way, without the bounds.
+//   phase-2 unit, Retained    1 to 4 groups of 16 retained channels x one quarter of the d outputs,
+//                             again as m16n8k16 tiles; h enters as a bf16 (high, low) pair in two
+//                             columns of the n dimension, so that y keeps fp32 accuracy.
+//   phase-2 unit, Candidate   the selected rows among 32 candidates (one word of the mask) x one
+//                             quarter of d: only selected rows are read, gathered by row id and
+//                             transposed by ldmatrix.
 //
-// Every consumer warp owns a private ring in shared memory that it fills with 16-byte
-// cp.async copies (each lane copies the very bytes it will read back as its mma A fragment: the
-// tiled layout stores fragments lane-contiguously) and drains NG-1 groups later.  A scheduler
-// warp claims units, waits for their dependencies and stages the small operands (h fragments,
-// selected row ids) so that consumer warps never poll global memory.
+// Phase 1 is dealt out statically (unit i of CTA c is unit c + i G); phase 2 is claimed from
+// per-quarter counters in shrinking chunks, which evens out what phase 1 left uneven.
 //
-// CTAs are pinned to a quarter of the output columns in phase 2 (they move to another quarter
-// when theirs is exhausted), partial y goes to an fp32 accumulator with vector reductions at L2;
-// the CTA that finishes last casts it, re-arms the counters and advances the epoch that
-// validates the flags.  Every wait is bounded; on expiry the kernel raises sync[SYNC_ERROR],
-// drains its copies and returns.
+// Warps of a CTA:
+//   8 consumer warps  each owns a private ring in shared memory that it fills with 16-byte cp.async
+//                     copies (each lane copies the very bytes it will read back as its mma A
+//                     fragment: the tiled layout stores fragments lane-contiguously) and drains
+//                     NG - 1 groups later; each covers 1/8 of the k range (phase 1) or of the
+//                     output columns of the quarter (phase 2).
+//   scheduler warp    deals out / claims units, waits for their dependencies and stages the small
+//                     operands (h fragments, selected row ids), so consumer warps never poll global memory.
+//   reducer warp      adds the consumer warps' partial sums of a phase-1 unit, applies the activation
+//                     and publishes h as 8-byte words (value, epoch of the step): a word carries its
+//                     own validity, so there are no ready flags and no fences on the consumer side.
+//   selection warp    the top-k of the candidates, replicated: every CTA computes the same mask from
+//                     the same streamed scores and keeps it in its own shared memory.  Candidates
+//                     whose streamed score is within the error bounds of the k-th are re-scored
+//                     exactly in fp64 (these jobs are dealt out over the CTAs), so the mask is the
+//                     one exact arithmetic gives.
+//
+// Partial y goes to an fp32 accumulator with vector reductions at L2; the CTA that finishes last
+// casts it, re-arms the counters and advances the epoch.  Every wait is bounded; on expiry the
+// kernel raises sync[SYNC_ERROR], drains its copies and returns.
 #include "pop_common.cuh"
 #include <stdlib.h>
 #include <string.h>
@@ -253,7 +264,7 @@ __device__ __noinline__ void refine_job(const StreamParams& P, int c, int e, int
 // stream weights never wait for another CTA's selection.  Only the fp64 re-scoring is shared out
 // (job e goes to CTA e mod G) and exchanged through global memory.
 //
-// The streamed scores a_i (fp32, P.keys32) are approximate, each with a bound m_i of its error
+// The streamed scores a_i (fp32, P.km) are approximate, each with a bound m_i of its error
 // (m = max m_i).  Let [tau_lo, tau_hi] be a bucket of key values that holds the k-th largest a_i.
 // a_i > tau_hi + 2m  => i is in the exact top-k (fewer than k candidates have a_j > tau_hi, and
 // every other one has an exact score below i's); a_i < tau_lo - 2m => i is not (the k candidates
@@ -829,7 +840,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     }
                 }
             }
-            if (is_cand) __threadfence();                    // keys and margins before the count below
+            if (is_cand) __threadfence();                    // h, scores and bounds before the count below
             __syncwarp();
             if (lane == 0) {
                 __threadfence_block();
@@ -1157,7 +1168,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         __syncthreads();
         if (tid == 0) {
             P.sync[SYNC_TICKET] = 0;
-            P.sync[SYNC_P1] = 0;
             P.sync[SYNC_CAND_DONE] = 0;
 #pragma unroll
             for (int q = 0; q < 4; ++q) { P.sync[SYNC_Q0 + 32 * q] = 0; P.sync[SYNC_QC0 + 32 * q] = 0; }
