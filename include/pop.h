@@ -114,6 +114,16 @@ int pop_partition_indices(const pop_partition_t* p, const int32_t** d_ret,
 /* Prefill importance scores I_i (Eq. 3), DEVICE double [N], owned by the partition. */
 int pop_partition_scores(const pop_partition_t* p, const double** d_scores);
 
+/*
+ * Diagnostic view of the last decode step's candidate scoring (Sec. 3.3 decoding stage) on a
+ * partition served by the streaming kernel: DEVICE array of n_cand pairs of fp32 values
+ * (score as streamed through the tensor cores, bound of |that score - exact score|), owned by
+ * the partition.  The selection treats a candidate as decided only when the bounds separate it
+ * from the k-th score, and re-scores the others exactly; tests use this view to check the bounds
+ * against exact arithmetic.  POP_ERR_UNSUPPORTED when the partition is served by another kernel.
+ */
+int pop_partition_streamed_scores(const pop_partition_t* p, const float** d_score_bound_pairs);
+
 /* Shape of a partition: any output may be NULL. */
 int pop_partition_shape(const pop_partition_t* p, int* d, int* N, pop_dtype_t* dtype);
 

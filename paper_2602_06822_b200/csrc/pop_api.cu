@@ -253,6 +253,13 @@ extern "C" int pop_partition_scores(const pop_partition_t* p, const double** d_s
     return POP_OK;
 }
 
+extern "C" int pop_partition_streamed_scores(const pop_partition_t* p, const float** d_score_bound_pairs) {
+    if (!p || !d_score_bound_pairs) return POP_ERR_INVALID_ARG;
+    if (p->layout != POP_LAYOUT_TILED) return POP_ERR_UNSUPPORTED;
+    *d_score_bound_pairs = reinterpret_cast<const float*>(p->keys);
+    return POP_OK;
+}
+
 extern "C" int pop_partition_shape(const pop_partition_t* p, int* d, int* N, pop_dtype_t* dtype) {
     if (!p) return POP_ERR_INVALID_ARG;
     if (d) *d = p->d;

@@ -55,6 +55,7 @@ SIGNATURES = {
     "pop_partition_sizes": (C.c_int, [_P] + [C.POINTER(C.c_int)] * 3),
     "pop_partition_indices": (C.c_int, [_P] + [C.POINTER(_P)] * 3),
     "pop_partition_scores": (C.c_int, [_P, C.POINTER(_P)]),
+    "pop_partition_streamed_scores": (C.c_int, [_P, C.POINTER(_P)]),
     "pop_partition_shape": (C.c_int, [_P, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "pop_partition_check": (C.c_int, [_P]),
     "pop_partition_destroy": (C.c_int, [_P]),
@@ -154,7 +155,7 @@ class Partition:
         """torch view (no copy) of a device array owned by the partition."""
         torch = _torch()
         if n == 0:
-            return torch.empty(0, device=self.device, dtype={"<i4": torch.int32, "<f8": torch.float64}[typestr])
+            return torch.empty(0, device=self.device, dtype={"<i4": torch.int32, "<f8": torch.float64, "<f4": torch.float32}[typestr])
         return torch.as_tensor(_DevView(ptr, n, typestr), device=self.device)
 
     def indices_device(self):
@@ -173,6 +174,14 @@ class Partition:
         p = C.c_void_p()
         _check(lib().pop_partition_scores(self.handle, C.byref(p)), "pop_partition_scores")
         return self._view(p.value, self.N, "<f8").cpu().numpy()
+
+    def streamed_scores(self):
+        """(score, bound) of every candidate as the streaming kernel's last step saw them: two host float32
+        arrays (synchronises); raises PopError(POP_ERR_UNSUPPORTED) for partitions served by another kernel."""
+        p = C.c_void_p()
+        _check(lib().pop_partition_streamed_scores(self.handle, C.byref(p)), "pop_partition_streamed_scores")
+        pairs = self._view(p.value, 2 * self.n_cand, "<f4").cpu().numpy().reshape(self.n_cand, 2)
+        return pairs[:, 0].copy(), pairs[:, 1].copy()
 
     def check(self):
         _check(lib().pop_partition_check(self.handle), "pop_partition_check")

@@ -35,6 +35,25 @@ def weights_host(w):
     return tuple(np.asarray(a.values, dtype=np.float64) for a in (w.weights.Wg, w.weights.Wu, w.weights.Wd))
 
 
+def check_streamed_bounds(part, o, k):
+    """Streaming kernel only: the bound it attaches to every streamed candidate score must cover the distance to
+    the exact score (the selection relies on it: Sec. 3.3 ranks by the exact scores), with room to spare."""
+    if part.n_cand == 0 or k <= 0 or k >= part.n_cand:
+        return                      # nothing is ranked: the kernel does not look at the scores
+    try:
+        a, m = part.streamed_scores()
+    except pop.PopError as e:
+        assert e.status == pop.POP_ERR_UNSUPPORTED
+        return                      # served by the fused / simple kernels, which score in fp64
+    exact = np.asarray(o["scores"], dtype=np.float64)
+    err = np.abs(a.astype(np.float64) - exact)
+    assert np.all(np.isfinite(m)) and np.all(m >= 0)
+    bad = err > m
+    assert not bad.any(), f"error bound violated for {int(bad.sum())} candidates (worst ratio {np.max(err / np.maximum(m, 1e-300)):.3g})"
+    # the bounds are meant to be loose by a wide factor (the model doubles the worst case twice)
+    assert np.max(err / np.maximum(m, 1e-300)) <= 0.25
+
+
 def run_decode_parity(w, part, R, C, steps, k, Wh):
     cfg = w.cfg
     dev = torch.device("cuda:0")
@@ -57,6 +76,7 @@ def run_decode_parity(w, part, R, C, steps, k, Wh):
             yref = po.masked_ffn(w.xs.values[t], *Wh, active)
         swaps += sw
         worst = max(worst, pr.rel_err(pr.host_values(y), yref))
+        check_streamed_bounds(part, o, k)
     part.check()
     assert worst <= pr.TOL[cfg.dtype], f"max relative output error {worst:.3e}"
     return worst, swaps
