@@ -151,23 +151,29 @@ extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg
     if (rc != POP_OK) return rc;
 
     // temporaries: column norms and activation energies, freed in stream order
-    double *norm = nullptr, *s2 = nullptr;
+    double *norm = nullptr, *s2 = nullptr, *s2part = nullptr;
+    const bool gemm = pop_prefill_s2_gemm_supported(d);
     cudaError_t e = cudaMallocAsync((void**)&norm, sizeof(double) * (size_t)N, st);
     if (e == cudaSuccess) e = cudaMallocAsync((void**)&s2, sizeof(double) * (size_t)N, st);
+    if (e == cudaSuccess && gemm)
+        e = cudaMallocAsync((void**)&s2part, sizeof(double) * (size_t)N * (size_t)pop_prefill_s2_gemm_splits(L), st);
     if (e != cudaSuccess) {
         pop_set_cuda_error(e, "cudaMallocAsync");
         if (norm) cudaFreeAsync(norm, st);
+        if (s2) cudaFreeAsync(s2, st);
         partition_free(p);
         return POP_ERR_ALLOC;
     }
     rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
-    if (rc == POP_OK) rc = pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
+    if (rc == POP_OK) rc = gemm ? pop_launch_prefill_s2_gemm(X, L, d, Wg, Wu, N, dtype, s2part, s2, st)
+                                : pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
     if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, p->scores, st);
     if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->idx_ret, p->idx_cand, p->idx_pruned, st);
     if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
                                                          : pop_launch_repack(p, Wg, Wu, Wd, norm, st);
     cudaFreeAsync(norm, st);
     cudaFreeAsync(s2, st);
+    if (s2part) cudaFreeAsync(s2part, st);
     if (rc != POP_OK) { cudaStreamSynchronize(st); partition_free(p); return rc; }
     *out = p;
     return POP_OK;

@@ -107,6 +107,11 @@ int pop_launch_colnorm(const void* Wd, int d, int N, pop_dtype_t dt, double* nor
 int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, const void* Wu, int N,
                                 pop_dtype_t dt, const int32_t* chan_list /*NULL = all*/, int n_list,
                                 double* s2 /*[N], entries of listed channels are overwritten*/, cudaStream_t st);
+// exact fp64 energies as a register-blocked GEMM (d a multiple of 16); s2part: [pop_prefill_s2_gemm_splits(L)][N] scratch
+bool pop_prefill_s2_gemm_supported(int d);
+int pop_prefill_s2_gemm_splits(int L);
+int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
+                               double* s2part, double* s2, cudaStream_t st);
 int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st);
 int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand,
                          int32_t* idx_ret, int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);

@@ -134,6 +134,197 @@ int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, con
     return POP_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same activation energy, exact in fp64, as a register-blocked GEMM for hidden sizes that
+// are a multiple of 16: the fp64 pipe, not shared memory or the conversions, is what bounds it.
+//
+// Block = 256 threads = 8 warps; block tile = 256 tokens x 32 channels (gate and up at once);
+// a warp owns 32 tokens x 32 channels, lane (tg, cg) = (lane / 8, lane % 8) a tile of 8 tokens x
+// 4 channels x {gate, up} = 64 accumulators.  K is consumed in chunks of 16, staged in shared
+// memory as doubles ([k][token] and [k][channel], so a lane reads its operands as contiguous
+// 16-byte pieces that the lanes of a warp share by broadcast), double-buffered with the next
+// chunk's global loads in flight during the arithmetic.  blockIdx.y splits the tokens into
+// ranges of tok_per_split; range y writes its partial energies to s2out[y * out_stride + channel],
+// and the caller adds the ranges in a fixed order.
+// ---------------------------------------------------------------------------------------------
+#define G2_TOK 256
+#define G2_CH 32
+#define G2_KT 16
+
+template <typename T>
+__global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
+    const T* __restrict__ X, int L, int d, const T* __restrict__ Wg, const T* __restrict__ Wu,
+    const int32_t* __restrict__ chan_list, int n_list, int tok_per_split, double* __restrict__ s2out, int out_stride) {
+    constexpr int EPV = 16 / sizeof(T);               // elements per 16-byte vector
+    constexpr int XV = G2_KT / EPV;                   // vectors per token row and chunk
+    constexpr int WV = 8 / EPV;                       // vectors per (matrix, channel, half chunk)
+    extern __shared__ __align__(16) double g2_sm[];
+    double* Xs = g2_sm;                               // [2][G2_KT][G2_TOK]
+    double* Gs = Xs + 2 * G2_KT * G2_TOK;             // [2][G2_KT][G2_CH]
+    double* Us = Gs + 2 * G2_KT * G2_CH;
+    __shared__ int chan[G2_CH];
+    __shared__ double red[8][G2_CH];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, tg = lane >> 3, cg = lane & 7;
+    const int c0 = blockIdx.x * G2_CH;
+    if (tid < G2_CH) {
+        const int li = c0 + tid;
+        chan[tid] = (li < n_list) ? (chan_list ? chan_list[li] : li) : -1;
+    }
+    __syncthreads();
+    const int t_begin = blockIdx.y * tok_per_split, t_end = min(L, t_begin + tok_per_split);
+    const int nk = d / G2_KT;
+
+    // staging roles: every thread one token row of X; threads 0..127 one (matrix, channel, half chunk) of W
+    const int wm = tid >> 6, wc = (tid >> 1) & 31, wh = tid & 1;
+    const int wch = tid < 128 ? chan[wc] : -1;
+    const T* wrow = wch >= 0 ? (wm ? Wu : Wg) + (size_t)wch * d + wh * 8 : nullptr;
+
+    double e[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int t0 = t_begin; t0 < t_end; t0 += G2_TOK) {
+        const int tok = t0 + tid;
+        const T* xrow = tok < t_end ? X + (size_t)tok * d : nullptr;
+        uint4 xr[XV], wr[WV];
+        auto fetch = [&](int kc) {
+#pragma unroll
+            for (int v = 0; v < XV; ++v)
+                xr[v] = xrow ? __ldg(reinterpret_cast<const uint4*>(xrow + kc * G2_KT) + v) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int v = 0; v < WV; ++v)
+                wr[v] = wrow ? __ldg(reinterpret_cast<const uint4*>(wrow + kc * G2_KT) + v) : make_uint4(0u, 0u, 0u, 0u);
+        };
+        auto stash = [&](int buf) {
+#pragma unroll
+            for (int v = 0; v < XV; ++v) {
+                float f[EPV];
+                Elem<T>::unpack(xr[v], f);
+#pragma unroll
+                for (int j = 0; j < EPV; ++j) Xs[(buf * G2_KT + v * EPV + j) * G2_TOK + tid] = (double)f[j];
+            }
+            if (tid < 128) {
+                double* dst = wm ? Us : Gs;
+#pragma unroll
+                for (int v = 0; v < WV; ++v) {
+                    float f[EPV];
+                    Elem<T>::unpack(wr[v], f);
+#pragma unroll
+                    for (int j = 0; j < EPV; ++j) dst[(buf * G2_KT + wh * 8 + v * EPV + j) * G2_CH + wc] = (double)f[j];
+                }
+            }
+        };
+        double g[8][4], u[8][4];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) { g[j][c] = 0.0; u[j][c] = 0.0; }
+
+        fetch(0);
+        stash(0);
+        __syncthreads();
+#pragma unroll 1
+        for (int kc = 0; kc < nk; ++kc) {
+            const int buf = kc & 1;
+            if (kc + 1 < nk) fetch(kc + 1);
+            const double* xs = Xs + (size_t)buf * G2_KT * G2_TOK + warp * 32 + tg * 8;
+            const double* gs = Gs + (size_t)buf * G2_KT * G2_CH + cg * 4;
+            const double* us = Us + (size_t)buf * G2_KT * G2_CH + cg * 4;
+#pragma unroll
+            for (int k = 0; k < G2_KT; ++k) {
+                double xv[8], gv[4], uv[4];
+#pragma unroll
+                for (int j = 0; j < 8; j += 2) {
+                    const double2 t2 = *reinterpret_cast<const double2*>(xs + k * G2_TOK + j);
+                    xv[j] = t2.x; xv[j + 1] = t2.y;
+                }
+#pragma unroll
+                for (int c = 0; c < 4; c += 2) {
+                    const double2 a2 = *reinterpret_cast<const double2*>(gs + k * G2_CH + c);
+                    const double2 b2 = *reinterpret_cast<const double2*>(us + k * G2_CH + c);
+                    gv[c] = a2.x; gv[c + 1] = a2.y; uv[c] = b2.x; uv[c + 1] = b2.y;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        g[j][c] = fma(gv[c], xv[j], g[j][c]);
+                        u[j][c] = fma(uv[c], xv[j], u[j][c]);
+                    }
+            }
+            if (kc + 1 < nk) stash(buf ^ 1);
+            __syncthreads();
+        }
+        // tokens past the end contribute silu(0) * 0 = 0
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const double h = silu_f64(g[j][c]) * u[j][c];
+                e[c] = fma(h, h, e[c]);
+            }
+    }
+    // channel sums: over the 4 token groups of the warp, then over the 8 warps, in a fixed order
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        e[c] += __shfl_xor_sync(0xffffffffu, e[c], 8);
+        e[c] += __shfl_xor_sync(0xffffffffu, e[c], 16);
+    }
+    if (tg == 0) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) red[warp][cg * 4 + c] = e[c];
+    }
+    __syncthreads();
+    if (tid < G2_CH && chan[tid] >= 0) {
+        double sum = 0.0;
+#pragma unroll 1
+        for (int r = 0; r < 8; ++r) sum += red[r][tid];
+        s2out[(size_t)blockIdx.y * out_stride + chan[tid]] = sum;
+    }
+}
+
+// s2[i] = sum over the token ranges (ascending) of s2part[y][i]
+__global__ void sum_ranges_kernel(const double* __restrict__ s2part, int nsplit, int N, double* __restrict__ s2) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    double sum = 0.0;
+    for (int y = 0; y < nsplit; ++y) sum += s2part[(size_t)y * N + i];
+    s2[i] = sum;
+}
+
+int pop_prefill_s2_gemm_splits(int L) { return L > 0 ? (L + G2_TOK - 1) / G2_TOK : 1; }
+
+bool pop_prefill_s2_gemm_supported(int d) { return d >= G2_KT && d % G2_KT == 0; }
+
+int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
+                               double* s2part, double* s2, cudaStream_t st) {
+    if (N <= 0) return POP_OK;
+    const int nsplit = pop_prefill_s2_gemm_splits(L);
+    const size_t smem = sizeof(double) * (2 * G2_KT * G2_TOK + 4 * G2_KT * G2_CH);
+    dim3 grd((N + G2_CH - 1) / G2_CH, nsplit);
+    static thread_local int cfg_dev[2] = {-1, -1};
+    int dev = 0;
+    POP_CUDA(cudaGetDevice(&dev));
+    if (dt == POP_F32) {
+        auto kern = prefill_s2_gemm_kernel<float>;
+        if (cfg_dev[0] != dev) {
+            POP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            cfg_dev[0] = dev;
+        }
+        kern<<<grd, 256, smem, st>>>((const float*)X, L, d, (const float*)Wg, (const float*)Wu, nullptr, N, G2_TOK, s2part, N);
+    } else {
+        auto kern = prefill_s2_gemm_kernel<__nv_bfloat16>;
+        if (cfg_dev[1] != dev) {
+            POP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            cfg_dev[1] = dev;
+        }
+        kern<<<grd, 256, smem, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu,
+                                     nullptr, N, G2_TOK, s2part, N);
+    }
+    POP_LAUNCHED();
+    sum_ranges_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2part, nsplit, N, s2);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
 // I_i = sqrt(s2_i) * n_i   (Eq. 3)
 __global__ void scores_kernel(const double* __restrict__ s2, const double* __restrict__ norm, int N,
                               double* __restrict__ scores) {
