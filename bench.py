@@ -168,6 +168,24 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------- multi-rank arithmetic
+def max_over_ranks(v, world, device):
+    """The slowest rank's time: every rank contributes its own device-measured duration."""
+    if world == 1:
+        return v
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([v], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, units_per_rank, max_ms):
+    """Replicas only (the path does not shard): every rank processes `units_per_rank` layer-steps of its own
+    seeded workload; the job's throughput is all of them over the slowest rank's time."""
+    return world * units_per_rank / (max_ms * 1e-3)
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def run_pop(args):
     import torch
@@ -280,11 +298,7 @@ def run_pop(args):
     e2e_steps = max(1, args.steps // 2)
 
     def reduce_max(v):
-        if world == 1:
-            return v
-        t = torch.tensor([v], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return max_over_ranks(v, world, dev)
 
     dec_ms = reduce_max(res["decode_ms"])
     pre_ms = reduce_max(res["prefill_ms"])
@@ -292,8 +306,8 @@ def run_pop(args):
     e2e_dec_ms = reduce_max(e2e["decode_ms"] + e2e["prefill_ms"])
     layer_steps = layers * tokens * args.steps
     us_per_ls = 1e3 * dec_ms / layer_steps
-    value = world * layer_steps / (dec_ms * 1e-3)
-    e2e_value = world * (layers * tokens * e2e_steps) / (e2e_dec_ms * 1e-3)
+    value = whole_job_value(world, layer_steps, dec_ms)
+    e2e_value = whole_job_value(world, layers * tokens * e2e_steps, e2e_dec_ms)
 
     if rank == 0:
         peaks = {}
