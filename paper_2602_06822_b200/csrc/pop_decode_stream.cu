@@ -82,7 +82,7 @@ struct StreamParams {
     uint8_t* mask_out;
     int32_t* sel_out;
     int d, B, k, n_ret, n_cand, n_rt, n_cg, n_ret_pad, h_stride;
-    int Uc, U1, n_cu, NG, NPB, p2_macro;
+    int Uc, U1, n_cu, NG, NPB, p2_macro, window;
     double cstep;                  // error bound of one warp's partial dot product / the largest magnitude in it
     int off_part, off_hfrag, off_rows, off_ystage, off_sel, off_ctrl;
 };
@@ -190,6 +190,18 @@ __device__ __forceinline__ u32 pack2(u32 lo, u32 hi) { return lo | (hi << 16); }
 __device__ __forceinline__ u64 h_word(float v, u32 epoch) { return (u64)__float_as_uint(v) | ((u64)epoch << 32); }
 
 #define POP_RAISE(code) do { ctrl->abort = 1; atomicExch(gerr, (u32)(code)); } while (0)
+
+// Polls an h word until it carries the epoch of this step (bounded; ok = false on expiry or abort).
+__device__ __noinline__ u64 poll_h(const u64* p, u32 epoch, Ctrl* ctrl, u32* gerr, bool& ok) {
+    u32 sp = 0;
+    for (;;) {
+        const u64 hw = __ldcg(p);
+        if ((u32)(hw >> 32) == epoch) return hw;
+        if (ctrl->abort) { ok = false; return 0ull; }
+        if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_FLAG); ok = false; return 0ull; }
+        __nanosleep(64);
+    }
+}
 
 // Event timestamps for performance work: compiled in only with -DPOP_STREAM_TRACE (a build of its own);
 // slot `id` of the calling CTA gets the time at which its lane 0 passed the marker.
@@ -555,7 +567,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     cm = min(cm, __shfl_xor_sync(0xffffffffu, cm, off));
                     cg = min(cg, __shfl_xor_sync(0xffffffffu, cg, off));
                 }
-                if (filled - cm < ND && sched_groups - cg < P.NG + 2 * MAXG) break;
+                if (filled - cm < ND && sched_groups - cg < P.NG + (stage == 0 ? 2 * MAXG : P.window)) break;
                 if (ctrl->abort) { ok = false; break; }
                 if (++spins > SPIN_LIMIT) { ctrl->abort = 1; atomicExch(gerr, (u32)ERR_THROTTLE); ok = false; break; }
                 __nanosleep(40);
@@ -656,46 +668,53 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             a = __shfl_sync(0xffffffffu, a, 0);
             b = __shfl_sync(0xffffffffu, b, 0);
             ng = __shfl_sync(0xffffffffu, ng, 0);
+            stage = __shfl_sync(0xffffffffu, stage, 0);      // the look-ahead test above is taken by all lanes
             if (type < 0) { ok = false; break; }
             const int dslot = filled % ND;
             if (type == T_P2_RET) {
-                // h of the unit's channels, as mma B fragments; a value not yet written this step (its
-                // epoch tag is old) is polled until the phase-1 unit that owns it has published it
-                for (int gi = 0; gi < ng && ok; ++gi) {
+                // h of the unit's channels, as mma B fragments.  All words of the unit are fetched at once (one
+                // memory round trip per unit); a word not yet written in this step (its epoch tag is old) is
+                // then polled until the phase-1 unit that owns it has published it.
+                u64 hw[MAXG][NBLK][4];
 #pragma unroll
-                    for (int nb = 0; nb < NBLK; ++nb) {
-                        const int n = g8 + 8 * nb, bb = n >> 1, part = n & 1;
-                        u32 b0 = 0, b1 = 0;
-                        if (bb < B) {
-                            const u64* hp = P.h + (size_t)bb * P.h_stride + 16 * (a + gi);
-                            float v[4];
-                            u32 sp = 0;
-                            for (;;) {
-                                bool all = true;
+                for (int gi = 0; gi < MAXG; ++gi)
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
-                                    if (16 * (a + gi) + kk < P.n_ret) {         // padding channels are zero
-                                        const u64 hw = __ldcg(hp + kk);
-                                        all = all && (u32)(hw >> 32) == epoch;
-                                        v[e] = __uint_as_float((u32)hw);
-                                    } else {
-                                        v[e] = 0.f;
-                                    }
-                                }
-                                if (all) break;
-                                if (ctrl->abort) { ok = false; break; }
-                                if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_FLAG); ok = false; break; }
-                                __nanosleep(64);
-                            }
-                            b0 = pack2(split_bits(v[0], part), split_bits(v[1], part));
-                            b1 = pack2(split_bits(v[2], part), split_bits(v[3], part));
+                    for (int nb = 0; nb < NBLK; ++nb)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int bb = (g8 + 8 * nb) >> 1;
+                            const int ch = 16 * (a + gi) + 2 * t4 + (e & 1) + (e >> 1) * 8;
+                            const bool live = gi < ng && bb < B && ch < P.n_ret;       // padding channels are zero
+                            hw[gi][nb][e] = live ? __ldcg(P.h + (size_t)bb * P.h_stride + ch) : ((u64)epoch << 32);
                         }
-                        hfrag[((dslot * MAXG + gi) * NBLK + nb) * 32 + lane] = make_uint2(b0, b1);
-                    }
-                }
+#pragma unroll
+                for (int gi = 0; gi < MAXG; ++gi)
+#pragma unroll
+                    for (int nb = 0; nb < NBLK; ++nb)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if ((u32)(hw[gi][nb][e] >> 32) != epoch) {
+                                const int bb = (g8 + 8 * nb) >> 1;
+                                const int ch = 16 * (a + gi) + 2 * t4 + (e & 1) + (e >> 1) * 8;
+                                hw[gi][nb][e] = poll_h(P.h + (size_t)bb * P.h_stride + ch, epoch, ctrl, gerr, ok);
+                            }
+                        }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+#pragma unroll
+                for (int gi = 0; gi < MAXG; ++gi)
+#pragma unroll
+                    for (int nb = 0; nb < NBLK; ++nb) {
+                        if (gi < ng) {
+                            const int part = (g8 + 8 * nb) & 1;
+                            float v[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) v[e] = __uint_as_float((u32)hw[gi][nb][e]);
+                            hfrag[((dslot * MAXG + gi) * NBLK + nb) * 32 + lane] =
+                                make_uint2(pack2(split_bits(v[0], part), split_bits(v[1], part)),
+                                           pack2(split_bits(v[2], part), split_bits(v[3], part)));
+                        }
+                    }
             } else if (type == T_P2_CAND) {
                 // row list of the unit: the selected ones among candidates 32 a .. 32 a + 31, padded with -1
                 const u32 m = ctrl->rowmask[a];
@@ -1297,6 +1316,10 @@ int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void
     P.U1 = P.Uc + p->n_rt;
     P.n_cu = k > 0 ? (p->n_cand + 31) / 32 : 0;
     P.p2_macro = p2_macro_env < 1 ? 1 : (p2_macro_env > MAXG ? MAXG : p2_macro_env);
+    // groups the scheduler may stage beyond the copy ring in phase 2: what is staged is committed to this CTA, so a
+    // deep queue makes the CTAs finish unevenly, a shallow one lets the ring run dry
+    static const int window_env = getenv("POP_P2_WINDOW") ? atoi(getenv("POP_P2_WINDOW")) : 2 * MAXG;
+    P.window = window_env < 1 ? 1 : (window_env > 2 * MAXG ? 2 * MAXG : window_env);
     const int gs = p->d / 1024;
     const int nblk = B <= 4 ? 1 : 2;
 #define POP_CASE(G_, N_) if (gs == G_ && nblk == N_) return launch_stream<G_, N_>(P, p, st);
