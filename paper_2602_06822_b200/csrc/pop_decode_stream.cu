@@ -99,6 +99,7 @@ struct Ctrl {
     volatile int cons_g[NCW];
     int cmt[NCW][8];               // consumer warps: commit index of each ring position
     float xmax[POP_MAX_BATCH];     // max |x[b][:]|
+    volatile int p1_started;       // phase-1 units the consumer warps have started (direct-load phase 1)
     volatile int sel_final;        // this CTA's copy of the selection (rowmask) is final
     u32 rowmask[KPL];              // bit l of word j: candidate 32 j + l is selected in this step
     u32 selsm[POP_SELECT_SMEM_WORDS(32)];
@@ -128,6 +129,12 @@ __device__ __forceinline__ void cp_wait_pending(int n) {      // n in [0, 7]
         case 6: cp_wait<6>(); break;
         default: cp_wait<7>(); break;
     }
+}
+__device__ __forceinline__ uint4 ldg_stream(const void* p) {       // read-once global data, not kept in L1
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
 }
 __device__ __forceinline__ uint4 lds128(u32 addr) {
     uint4 v;
@@ -528,7 +535,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
 
     if (tid == 0) {
         ctrl->filled = 0; ctrl->abort = 0; ctrl->reduced = 0; ctrl->last = 0;
-        ctrl->sel_final = 0;
+        ctrl->sel_final = 0; ctrl->p1_started = 0;
         for (int b = 0; b < NPB_MAX; ++b) mbar_init(smem_u32(&ctrl->bar_full[b]), NCW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -547,7 +554,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
     if (warp == W_SCHED) {
         // ================================================================= scheduler warp
         const u32 epoch = ld_acquire_gpu(P.sync + SYNC_EPOCH) + 1u;
-        int stage = 0, nstatic = 0, qoff = 0, pend_lo = 0, pend_hi = 0, pend_q = 0;   // lane 0's state
+        int stage = 1, qoff = 0, pend_lo = 0, pend_hi = 0, pend_q = 0;   // lane 0's state (stage 1: retained groups, 2: what is left of the candidate units)
         bool sel_waited = false;
         int spec_amt = 0, cand_exh = 0;     // cand_exh bit q: the candidate units of quarter q are all claimed
         const int cpq = (G + 3) >> 2;      // CTAs that start on the same quarter
@@ -556,6 +563,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         int filled = 0, sched_groups = 0;
         const int myq = cta & 3;
         bool done = false, ok = true;
+        {
+            // Phase 2 is claimed dynamically, and what is claimed is committed to this CTA: the first claim waits
+            // until the consumer warps are two units from the end of their phase 1, late enough to see which
+            // CTAs are ahead, early enough for the first descriptors to be staged when they get there.
+            const int p1_count = cta < P.U1 ? (P.U1 - cta + G - 1) / G : 0;
+            u32 sp = 0;
+            while (ctrl->p1_started < p1_count - 1) {
+                if (ctrl->abort) { ok = false; break; }
+                if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_THROTTLE); ok = false; break; }
+                __nanosleep(200);
+            }
+        }
         while (!done && ok) {
             // room in the descriptor ring and in the look-ahead window?
             u32 spins = 0;
@@ -567,7 +586,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     cm = min(cm, __shfl_xor_sync(0xffffffffu, cm, off));
                     cg = min(cg, __shfl_xor_sync(0xffffffffu, cg, off));
                 }
-                if (filled - cm < ND && sched_groups - cg < P.NG + (stage == 0 ? 2 * MAXG : P.window)) break;
+                if (filled - cm < ND && sched_groups - cg < P.NG + P.window) break;
                 if (ctrl->abort) { ok = false; break; }
                 if (++spins > SPIN_LIMIT) { ctrl->abort = 1; atomicExch(gerr, (u32)ERR_THROTTLE); ok = false; break; }
                 __nanosleep(40);
@@ -581,19 +600,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         ng = pend_hi - pend_lo;
                         type = T_P2_RET; a = pend_lo; b = pend_q; pend_lo += ng;
                         break;
-                    }
-                    if (stage == 0) {
-                        // phase 1 is dealt out statically (unit i of this CTA = cta + i G: no claim latency);
-                        // phase 2, claimed dynamically below, evens out what that leaves
-                        const int p = cta + nstatic * G;
-                        ++nstatic;
-                        if (p < P.U1) {
-                            if (p < P.Uc) { type = T_P1_CAND; a = p; } else { type = T_P1_RET; a = p - P.Uc; }
-                            ng = MAXG;
-                            break;
-                        }
-                        stage = 1;
-                        POP_TRACE(7);
                     }
                     if (stage == 1) {
                         // retained groups of this CTA's quarter, then what is left of the other quarters
@@ -668,7 +674,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             a = __shfl_sync(0xffffffffu, a, 0);
             b = __shfl_sync(0xffffffffu, b, 0);
             ng = __shfl_sync(0xffffffffu, ng, 0);
-            stage = __shfl_sync(0xffffffffu, stage, 0);      // the look-ahead test above is taken by all lanes
             if (type < 0) { ok = false; break; }
             const int dslot = filled % ND;
             if (type == T_P2_RET) {
@@ -920,11 +925,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                 idesc = ctrl->desc[im % ND];
                 ihave = true; ig = 0;
                 // this lane's source address of the unit's first group and the step from group to group
-                if (idesc.x <= T_P1_RET) {
-                    const int tile = idesc.x == T_P1_RET ? idesc.y : P.n_rt + idesc.y;     // candidate tiles follow the retained ones
-                    isrc = P.GUt + ((size_t)tile * KT + (size_t)(w * S)) * SLOT + lane * 16;
-                    istep = GSL * SLOT;
-                } else if (idesc.x == T_P2_RET) {
+                if (idesc.x == T_P2_RET) {
                     isrc = P.WdTt + (((size_t)idesc.z * P.n_cg + (size_t)idesc.y) * (size_t)(KT >> 2) + (size_t)(w * GSL)) * SLOT + lane * 16;
                     istep = (KT >> 2) * SLOT;
                 }
@@ -973,17 +974,115 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             return base;
         };
 
-        // prologue: NG - 1 commits, group i in commit i when its descriptor is there.  Only the
-        // first group may block: a later unit's descriptor can depend on work this very CTA
-        // still has to do (a selected-candidate unit waits for the selection, which waits for
-        // every candidate unit), so the consumer side never waits for more than the group it
-        // is about to read.
-        for (int i = 0; i < NG - 1 && ok; ++i) {
-            if (!iend && icount <= i) {
-                issue_one(i == 0);
+        // The partial-sum buffer of phase-1 unit number p1seq must have been released by the reducer.
+        auto part_buffer_free = [&]() -> bool {
+            u32 sp = 0;
+            while (ctrl->reduced < p1seq - NPB + 1) {
+                if (ctrl->abort) return false;
+                if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_PART_FREE); return false; }
+                __nanosleep(20);
             }
-            cp_commit();
-            ++ncommit;
+            return true;
+        };
+        // Hands the partial sums (and, for a candidate unit, the magnitudes) of this warp's k range of a
+        // phase-1 unit to the reducer warp: [16 rows][BCAP columns] each.
+        auto deposit = [&](int type, int unit, const float (&c)[4], const float (&cmx)[4]) -> bool {
+            if (!part_buffer_free()) return false;
+            const int buf = p1seq % NPB;
+            float* pw = reinterpret_cast<float*>(smem + P.off_part) + ((size_t)buf * NCW + w) * PART_W;
+            if (2 * t4 < BCAP) {
+                pw[g8 * BCAP + 2 * t4] = c[0];
+                pw[g8 * BCAP + 2 * t4 + 1] = c[1];
+                pw[(g8 + 8) * BCAP + 2 * t4] = c[2];
+                pw[(g8 + 8) * BCAP + 2 * t4 + 1] = c[3];
+                if (type == T_P1_CAND) {
+                    float* mw = pw + 16 * BCAP;
+                    mw[g8 * BCAP + 2 * t4] = cmx[0];
+                    mw[g8 * BCAP + 2 * t4 + 1] = cmx[1];
+                    mw[(g8 + 8) * BCAP + 2 * t4] = cmx[2];
+                    mw[(g8 + 8) * BCAP + 2 * t4 + 1] = cmx[3];
+                }
+            }
+            if (tid == 0) ctrl->part_hdr[buf] = make_int2(type, unit);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->bar_full[buf]));
+            ++p1seq;
+            return true;
+        };
+
+        // Fills the copy ring for the descriptor-driven units: NG - 1 commits, group i in commit i when its
+        // descriptor is there.  block_first: the first group may wait for its descriptor; a later one never does:
+        // a later unit's descriptor can depend on work this very CTA still has to do (a selected-candidate
+        // unit waits for the selection, which waits for every candidate unit), so the consumer side never waits
+        // for more than the group it is about to read.
+        auto ring_prologue = [&](bool block_first) {
+            for (int i = 0; i < NG - 1 && ok; ++i) {
+                if (!iend && icount <= i) issue_one(block_first && i == 0);
+                cp_commit();
+                ++ncommit;
+            }
+        };
+
+        {
+            // ---- phase 1 on direct loads: unit i of this CTA is unit cta + i G; this warp's part of it is a
+            // contiguous run of S 512-byte slots, each lane's 16 bytes being its mma A fragment.
+            // Loads are issued in batches of BS slots into two register buffers that take turns: a batch is
+            // consumed (BS mma) and its buffer refilled at once with the batch after next, so BS to 2 BS loads
+            // per lane are in flight at any time.
+            constexpr int BS = S % 16 == 0 ? 8 : 5;
+            constexpr int NB = S / BS;
+            static_assert(S % BS == 0 && NB % 2 == 0, "a unit must be an even number of batches");
+            const int p1_count = cta < P.U1 ? (P.U1 - cta + G - 1) / G : 0;
+            auto src_of = [&](int i) -> const unsigned char* {
+                const int p = cta + i * G;
+                const int tile = p < P.Uc ? P.n_rt + p : p - P.Uc;        // candidate tiles follow the retained ones
+                return P.GUt + ((size_t)tile * KT + (size_t)(w * S)) * SLOT + lane * 16;
+            };
+            uint4 bufA[BS], bufB[BS];
+            if (p1_count > 0) {
+                const unsigned char* s0 = src_of(0);
+#pragma unroll
+                for (int j = 0; j < BS; ++j) bufA[j] = ldg_stream(s0 + j * SLOT);
+#pragma unroll
+                for (int j = 0; j < BS; ++j) bufB[j] = ldg_stream(s0 + (BS + j) * SLOT);
+            }
+#pragma unroll 1
+            for (int i = 0; i < p1_count && ok; ++i) {
+                if (w == 0 && lane == 0) ctrl->p1_started = i + 1;
+                if (i == p1_count - 1) ring_prologue(false);       // phase 2's first copies fly during the last unit
+                const int p = cta + i * G;
+                const bool is_cand = p < P.Uc;
+                const unsigned char* cur = src_of(i);
+                const unsigned char* nxt = i + 1 < p1_count ? src_of(i + 1) : nullptr;
+                float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
+                float cmx[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int b = 0; b < NB; ++b) {
+                    uint4 (&buf)[BS] = (b & 1) ? bufB : bufA;
+#pragma unroll
+                    for (int j = 0; j < BS; ++j) {
+                        const int sl = b * BS + j;
+                        if (sl & 1) mma_bf16(c2, buf[j], xf[sl][0], xf[sl][1]);
+                        else mma_bf16(c, buf[j], xf[sl][0], xf[sl][1]);
+                        if (is_cand) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) cmx[e] = fmaxf(cmx[e], fmaxf(fabsf(c[e]), fabsf(c2[e])));
+                        }
+                    }
+                    // refill with the batch after next: of this unit, or of the next one
+                    if (b + 2 < NB) {
+#pragma unroll
+                        for (int j = 0; j < BS; ++j) buf[j] = ldg_stream(cur + ((b + 2) * BS + j) * SLOT);
+                    } else if (nxt) {
+#pragma unroll
+                        for (int j = 0; j < BS; ++j) buf[j] = ldg_stream(nxt + ((b + 2 - NB) * BS + j) * SLOT);
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) c[e] += c2[e];
+                if (!deposit(is_cand ? T_P1_CAND : T_P1_RET, is_cand ? p : p - P.Uc, c, cmx)) { ok = false; break; }
+            }
+            if (p1_count == 0) ring_prologue(true);
         }
 
         // phase-2 accumulators: [m-tile][n-block][4]
@@ -1020,17 +1119,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             }
         };
 
-        // The partial-sum buffer of phase-1 unit number p1seq must have been released by the reducer.
-        auto part_buffer_free = [&]() -> bool {
-            u32 sp = 0;
-            while (ctrl->reduced < p1seq - NPB + 1) {
-                if (ctrl->abort) return false;
-                if (++sp > SPIN_LIMIT) { POP_RAISE(ERR_PART_FREE); return false; }
-                __nanosleep(20);
-            }
-            return true;
-        };
-
         while (ok) {
             // descriptor of the unit to consume
             {
@@ -1046,16 +1134,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             const int4 cd = ctrl->desc[cm % ND];
             const int dslot = cm % ND;
             if (cd.x == T_END) break;
-            const bool is_p1 = cd.x <= T_P1_RET, is_cand = cd.x == T_P1_CAND;
 #ifdef POP_STREAM_TRACE
             if (w == 0 && cd.x == T_P2_RET && cq < 0) POP_TRACE(11);
             if (w == 0 && cd.x == T_P2_CAND && !g_trace[cta * TRACE_SLOTS + 12]) POP_TRACE(12);
 #endif
 
             // ---- unit prologue
-            float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
-            float cmx[4] = {0.f, 0.f, 0.f, 0.f};              // candidate units: largest |accumulator| seen (either chain)
-            if (!is_p1 && cd.z != cq) {
+            if (cd.z != cq) {
                 if (cq >= 0) {
                     flush(cq);
 #pragma unroll
@@ -1079,25 +1164,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                     uint4 av[GSL];
 #pragma unroll
                     for (int j = 0; j < GSL; ++j) av[j] = lds128(base + lane * 16 + j * SLOT);
-                    if (is_p1) {
-                        // x fragments of group gi live in registers: static indices need the switch
-                        switch (gi) {
-#define POP_P1_GROUP(Q)                                                                                       \
-                            case Q:                                                                               \
-                                _Pragma("unroll") for (int j = 0; j < GSL; ++j) {                                 \
-                                    if (j & 1) mma_bf16(c2, av[j], xf[Q * GSL + j][0], xf[Q * GSL + j][1]);       \
-                                    else mma_bf16(c, av[j], xf[Q * GSL + j][0], xf[Q * GSL + j][1]);              \
-                                    if (is_cand) {                                                                \
-                                        _Pragma("unroll") for (int e = 0; e < 4; ++e)                             \
-                                            cmx[e] = fmaxf(cmx[e], fmaxf(fabsf(c[e]), fabsf(c2[e])));             \
-                                    }                                                                             \
-                                }                                                                                 \
-                                break;
-                            POP_P1_GROUP(0) POP_P1_GROUP(1) POP_P1_GROUP(2) POP_P1_GROUP(3)
-#undef POP_P1_GROUP
-                            default: break;
-                        }
-                    } else {
+                    {
                         uint2 hb[NBLK];
 #pragma unroll
                         for (int nb = 0; nb < NBLK; ++nb) hb[nb] = lds64(hf0 + (u32)((gi * NBLK + nb) * 32) * 8u);
@@ -1129,33 +1196,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             }
             if (!ok) break;
 
-            // ---- unit epilogue
-            if (is_p1) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) c[e] += c2[e];
-                // deposit the partial sums (and, for a candidate unit, the magnitudes) of this warp's k
-                // range for the reducer warp: [16 rows][BCAP columns] each
-                if (!part_buffer_free()) { ok = false; break; }
-                const int buf = p1seq % NPB;
-                float* pw = reinterpret_cast<float*>(smem + P.off_part) + ((size_t)buf * NCW + w) * PART_W;
-                if (2 * t4 < BCAP) {
-                    pw[g8 * BCAP + 2 * t4] = c[0];
-                    pw[g8 * BCAP + 2 * t4 + 1] = c[1];
-                    pw[(g8 + 8) * BCAP + 2 * t4] = c[2];
-                    pw[(g8 + 8) * BCAP + 2 * t4 + 1] = c[3];
-                    if (is_cand) {
-                        float* mw = pw + 16 * BCAP;
-                        mw[g8 * BCAP + 2 * t4] = cmx[0];
-                        mw[g8 * BCAP + 2 * t4 + 1] = cmx[1];
-                        mw[(g8 + 8) * BCAP + 2 * t4] = cmx[2];
-                        mw[(g8 + 8) * BCAP + 2 * t4 + 1] = cmx[3];
-                    }
-                }
-                if (tid == 0) ctrl->part_hdr[buf] = make_int2(cd.x, cd.y);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->bar_full[buf]));
-                ++p1seq;
-            }
             ++cm;
             if (lane == 0) ctrl->cons_m[w] = cm;
         }
