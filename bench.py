@@ -168,6 +168,19 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------- measured DRAM traffic
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture summarised in
+# profiles/pop_decode_stream_kernel_llama2_7b_r20_b1.md (226.05 MB read + 9.2 MB written).  Valid for the default
+# decode kernel of that workload only; None for anything else, and to be reset to None when that kernel changes.
+NCU_TRAFFIC_BYTES = {"llama2_7b_ffn_r20_b1": 235.3e6}
+
+
+def ncu_traffic(workload):
+    if os.environ.get("POP_DECODE_IMPL", "stream") not in ("", "stream"):
+        return None
+    return NCU_TRAFFIC_BYTES.get(workload)
+
+
 # ----------------------------------------------------------------------------- multi-rank arithmetic
 def max_over_ranks(v, world, device):
     """The slowest rank's time: every rank contributes its own device-measured duration."""
@@ -340,7 +353,7 @@ def run_pop(args):
                             "copied out and the stream synchronised"},
             "gpu_launches": int(res["launches"]),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_source": peak_src, "algorithmic_bytes_per_launch": abytes,
+                         "traffic": ncu_traffic(name), "peak_source": peak_src, "algorithmic_bytes_per_launch": abytes,
                          "frac_of_nominal_8TBs": achieved / 8000.0,
                          "kernel": "decode layer-step (all kernels of one pop_decode_step, averaged over the decode region)"},
         }
