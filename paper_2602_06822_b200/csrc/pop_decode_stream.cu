@@ -19,13 +19,15 @@
 // per-quarter counters in shrinking chunks, which evens out what phase 1 left uneven.
 //
 // Warps of a CTA:
-//   8 consumer warps  each owns a private ring in shared memory that it fills with 16-byte cp.async
-//                     copies (each lane copies the very bytes it will read back as its mma A
-//                     fragment: the tiled layout stores fragments lane-contiguously) and drains
-//                     NG - 1 groups later; each covers 1/8 of the k range (phase 1) or of the
-//                     output columns of the quarter (phase 2).
-//   scheduler warp    deals out / claims units, waits for their dependencies and stages the small
-//                     operands (h fragments, selected row ids), so consumer warps never poll global memory.
+//   8 consumer warps  each covers 1/8 of the k range (phase 1) or of the output columns of the quarter
+//                     (phase 2).  The tiled layout stores mma A fragments lane-contiguously, so in
+//                     phase 1 a lane's 16-byte global load IS its fragment: weights go from HBM to
+//                     registers to the tensor core, two batches of loads per lane taking turns.  In
+//                     phase 2 each warp owns a private ring in shared memory that it fills with
+//                     16-byte cp.async copies and drains NG - 1 groups later (gathered candidate rows
+//                     need shared memory anyway: they are transposed by ldmatrix).
+//   scheduler warp    claims phase-2 units, waits for their dependencies and stages the small operands
+//                     (h fragments, selected row ids), so consumer warps never poll global memory.
 //   reducer warp      adds the consumer warps' partial sums of a phase-1 unit, applies the activation
 //                     and publishes h as 8-byte words (value, epoch of the step): a word carries its
 //                     own validity, so there are no ready flags and no fences on the consumer side.
