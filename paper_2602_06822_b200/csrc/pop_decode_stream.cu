@@ -101,6 +101,7 @@ struct Ctrl {
     volatile int cons_g[NCW];
     int cmt[NCW][8];               // consumer warps: commit index of each ring position
     float xmax[POP_MAX_BATCH];     // max |x[b][:]|
+    u32 epoch;                     // epoch of this step (set by the scheduler warp)
     volatile int p1_started;       // phase-1 units the consumer warps have started (direct-load phase 1)
     volatile int sel_final;        // this CTA's copy of the selection (rowmask) is final
     u32 rowmask[KPL];              // bit l of word j: candidate 32 j + l is selected in this step
@@ -165,9 +166,6 @@ __device__ __forceinline__ u32 ld_acquire_gpu(const u32* p) {
     u32 v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
-}
-__device__ __forceinline__ void st_release_gpu(u32* p, u32 v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -556,6 +554,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
     if (warp == W_SCHED) {
         // ================================================================= scheduler warp
         const u32 epoch = ld_acquire_gpu(P.sync + SYNC_EPOCH) + 1u;
+        if (lane == 0) ctrl->epoch = epoch;
         int stage = 1, qoff = 0, pend_lo = 0, pend_hi = 0, pend_q = 0;   // lane 0's state (stage 1: retained groups, 2: what is left of the candidate units)
         bool sel_waited = false;
         int spec_amt = 0, cand_exh = 0;     // cand_exh bit q: the candidate units of quarter q are all claimed
@@ -1217,7 +1216,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
     }
     __syncthreads();
     if (ctrl->last) {
-        // every CTA has added its partial sums: cast, clear the accumulator, re-arm the counters
+        // every CTA has added its partial sums and is past its last use of the counters: re-arm them, advance the
+        // epoch (plain stores: the next launch on the stream starts only after this grid has completed), cast the
+        // accumulator and clear it
+        if (tid == 0) {
+            P.sync[SYNC_TICKET] = 0;
+            P.sync[SYNC_CAND_DONE] = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { P.sync[SYNC_Q0 + 32 * q] = 0; P.sync[SYNC_QC0 + 32 * q] = 0; }
+            P.sync[SYNC_RF_DONE] = 0;
+            P.sync[SYNC_EPOCH] = ctrl->epoch;
+        }
         float4* ya = reinterpret_cast<float4*>(P.y_acc);
         uint2* yo = reinterpret_cast<uint2*>(P.y);
 #pragma unroll 4
@@ -1225,17 +1234,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             const float4 v = __ldcg(ya + i);
             yo[i] = make_uint2(pack2(split_bits(v.x, 0), split_bits(v.y, 0)), pack2(split_bits(v.z, 0), split_bits(v.w, 0)));
             ya[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        __syncthreads();
-        if (tid == 0) {
-            P.sync[SYNC_TICKET] = 0;
-            P.sync[SYNC_CAND_DONE] = 0;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { P.sync[SYNC_Q0 + 32 * q] = 0; P.sync[SYNC_QC0 + 32 * q] = 0; }
-            P.sync[SYNC_RF_DONE] = 0;
-            const u32 epoch = P.sync[SYNC_EPOCH] + 1u;
-            __threadfence();
-            st_release_gpu(P.sync + SYNC_EPOCH, epoch);
         }
         if (warp == 0) POP_TRACE(18);
     }
