@@ -103,7 +103,9 @@ struct Ctrl {
     float xmax[POP_MAX_BATCH];     // max |x[b][:]|
     u32 epoch;                     // epoch of this step (set by the scheduler warp)
     volatile int p1_started;       // phase-1 units the consumer warps have started (direct-load phase 1)
+    volatile int sel_ready;        // rowmask holds the candidates decided by the streamed scores; umask marks the open words
     volatile int sel_final;        // this CTA's copy of the selection (rowmask) is final
+    u32 umask[KPL];                // bit l of word j: candidate 32 j + l awaits its exact score
     u32 rowmask[KPL];              // bit l of word j: candidate 32 j + l is selected in this step
     u32 selsm[POP_SELECT_SMEM_WORDS(32)];
 };
@@ -420,11 +422,15 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, u
             const u32 bu = __ballot_sync(0xffffffffu, is_un);
             const u32 bi = __ballot_sync(0xffffffffu, is_in);
             if (is_un) ulist[nu + __popc(bu & lt)] = i;
-            if (lane == 0) rowmask[j] = bi;
+            if (lane == 0) { rowmask[j] = bi; ctrl->umask[j] = bu; }
             nu += __popc(bu);
             nin += __popc(bi);
         }
+        // The words of the mask without an open candidate are final already: the scheduler may hand them out
+        // while the few open candidates are re-scored.
+        __threadfence_block();
         __syncwarp();
+        if (lane == 0) ctrl->sel_ready = 1;
         POP_TRACE(2);
         POP_TRACE_VALUE(16, nu);
         if (nu > 0) {
@@ -535,7 +541,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
 
     if (tid == 0) {
         ctrl->filled = 0; ctrl->abort = 0; ctrl->reduced = 0; ctrl->last = 0;
-        ctrl->sel_final = 0; ctrl->p1_started = 0;
+        ctrl->sel_final = 0; ctrl->sel_ready = 0; ctrl->p1_started = 0;
         for (int b = 0; b < NPB_MAX; ++b) mbar_init(smem_u32(&ctrl->bar_full[b]), NCW);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -558,6 +564,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         int stage = 1, qoff = 0, pend_lo = 0, pend_hi = 0, pend_q = 0;   // lane 0's state (stage 1: retained groups, 2: what is left of the candidate units)
         bool sel_waited = false;
         int spec_amt = 0, cand_exh = 0;     // cand_exh bit q: the candidate units of quarter q are all claimed
+        constexpr int NDEFER = 16;
+        int defer[NDEFER], ndefer = 0;      // claimed candidate units (word | quarter << 16) that wait for the final mask
         const int cpq = (G + 3) >> 2;      // CTAs that start on the same quarter
         u32 spec = 0;                      // result of a claim issued ahead of its use
         bool spec_valid = false;
@@ -610,10 +618,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         // than at the very end.
                         {
                             const int q = (myq + qoff) & 3;
-                            if (P.n_cu > 0 && !((cand_exh >> q) & 1) && ctrl->sel_final) {
+                            if (P.n_cu > 0 && !((cand_exh >> q) & 1) && ndefer < NDEFER && (ctrl->sel_final || ctrl->sel_ready)) {
                                 __threadfence_block();
                                 const int pc = (int)atomicAdd(P.sync + SYNC_QC0 + 32 * q, 1u);
                                 if (pc < P.n_cu) {
+                                    if (!ctrl->sel_final && ctrl->umask[pc] != 0u) {
+                                        defer[ndefer++] = pc | (q << 16);      // a word with an open candidate: after the final mask
+                                        continue;
+                                    }
                                     const int cnt = __popc(ctrl->rowmask[pc]);
                                     if (cnt == 0) continue;
                                     type = T_P2_CAND; a = pc; b = q; ng = (cnt + 15) >> 4;
@@ -642,8 +654,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         }
                         continue;
                     }
-                    // stage 2: selected candidate rows, one unit = one word of the mask (32 candidates), last of all
-                    if (qoff >= 4 || P.n_cu == 0) { type = T_END; break; }
+                    // stage 2: the candidate units left: those put off, then what nobody has claimed
+                    if (P.n_cu == 0 || (qoff >= 4 && ndefer == 0)) { type = T_END; break; }
                     if (!sel_waited) {
                         u32 sp = 0;
                         while (!ctrl->sel_final) {
@@ -655,6 +667,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         __threadfence_block();
                         sel_waited = true;
                         POP_TRACE(9);
+                    }
+                    if (ndefer > 0) {
+                        const int pq = defer[--ndefer];
+                        const int pc = pq & 0xffff;
+                        const int cnt = __popc(ctrl->rowmask[pc]);
+                        if (cnt == 0) continue;
+                        type = T_P2_CAND; a = pc; b = pq >> 16; ng = (cnt + 15) >> 4;
+                        break;
                     }
                     const int q = (myq + qoff) & 3;
                     if ((cand_exh >> q) & 1) { ++qoff; continue; }
