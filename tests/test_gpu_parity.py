@@ -320,3 +320,74 @@ def test_moe_small():
 def test_config4_moe_full_size():
     cfg = wl.config4_expert(0.2)
     run_moe_case(cfg, n_experts=8, steps=2)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("d,dtype", [(2048, wl.BF16), (128, wl.F32)])
+def test_all_candidate_scores_equal(d, dtype):
+    """x = 0 makes every candidate score 0: nothing separates the candidates, so the top-k is decided by the
+    tie-break alone (lowest channel ids, Sec. 3.3 ranking read as a total order) and y is exactly 0.  In the
+    streaming kernel this is the case where no candidate is decided by the streamed scores."""
+    cfg = wl.FFNConfig("zeros", d=d, N=384, dtype=dtype, prompt_tokens=16, decode_steps=1,
+                       ratios=wl.Ratios(0.4, 0.35, 0.25), seed=5)
+    w = wl.make_ffn_workload(cfg)
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, cfg.ratios.astuple())
+    R, C, _ = part.indices()
+    x0 = np.zeros_like(w.xs.values[0])
+    x = torch.zeros_like(pr.to_dev(w.xs, index=0))
+    for k in (1, part.n_cand // 2, part.n_cand - 1):
+        mask = torch.full((part.n_cand,), 9, dtype=torch.uint8, device="cuda:0")
+        sel = torch.full((k,), -1, dtype=torch.int32, device="cuda:0")
+        y = pop.decode_step(part, x, k, mask_out=mask, sel_out=sel)
+        torch.cuda.synchronize()
+        part.check()
+        o = po.decode_step(x0, *Wh, R, C, k)
+        assert np.array_equal(o["sel"], C[:k])                       # the oracle's own tie-break, stated
+        assert np.array_equal(sel.cpu().numpy(), o["sel"])
+        assert np.array_equal(mask.cpu().numpy(), o["mask"])
+        assert float(y.float().abs().max()) == 0.0
+    part.destroy()
+
+
+_LAUNCH_MODE_SCRIPT = r"""
+import sys
+import numpy as np, torch
+sys.path.insert(0, {root!r})
+from oracle import pop_oracle as po
+from paper_2602_06822_b200 import pop, workloads as wl
+from tests import parity as pr
+cfg = wl.FFNConfig("modes", d=2048, N=1536, dtype=wl.BF16, prompt_tokens=24, decode_steps=3,
+                   ratios=wl.Ratios(0.5, 0.25, 0.25), seed=11)
+w = wl.make_ffn_workload(cfg)
+Wh = tuple(np.asarray(a.values, dtype=np.float64) for a in (w.weights.Wg, w.weights.Wu, w.weights.Wd))
+Wg, Wu, Wd = (pr.to_dev(a) for a in (w.weights.Wg, w.weights.Wu, w.weights.Wd))
+part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, cfg.ratios.astuple())
+part.streamed_scores()          # raises unless the streaming kernel serves this partition
+R, C, _ = part.indices()
+k = part.n_cand // 2
+mask = torch.zeros(part.n_cand, dtype=torch.uint8, device="cuda:0")
+for t in range(3):
+    y = pop.decode_step(part, pr.to_dev(w.xs, index=t), k, mask_out=mask)
+    torch.cuda.synchronize()
+    part.check()
+    o = po.decode_step(w.xs.values[t], *Wh, R, C, k)
+    assert np.array_equal(mask.cpu().numpy(), o["mask"])
+    assert pr.rel_err(pr.host_values(y), o["y"]) <= pr.TOL[wl.BF16]
+print("mode ok")
+"""
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode", ["pdl", "coop", "plain"])
+def test_streaming_kernel_launch_modes(mode, decode_impl):
+    """The launch mode of the streaming kernel is read once per process, so each mode runs in a process of its own."""
+    if decode_impl != "stream":
+        pytest.skip("launch modes belong to the streaming kernel")
+    import os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, POP_STREAM_LAUNCH=mode, POP_DECODE_IMPL="stream")
+    out = subprocess.run([sys.executable, "-c", _LAUNCH_MODE_SCRIPT.format(root=root)], env=env, cwd=root,
+                         capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "mode ok" in out.stdout, out.stdout[-2000:] + out.stderr[-2000:]
