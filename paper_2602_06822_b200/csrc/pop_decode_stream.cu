@@ -616,6 +616,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         // Once the selection is final, the selected candidate rows of the quarter this CTA works on
                         // come first: they are small gathered units, better placed where retained groups follow
                         // than at the very end.
+                        if (ndefer > 0 && ctrl->sel_final) {
+                            // a unit put off for its open candidates: the mask is final now
+                            __threadfence_block();
+                            const int pq = defer[--ndefer];
+                            const int pc = pq & 0xffff;
+                            const int cnt = __popc(ctrl->rowmask[pc]);
+                            if (cnt == 0) continue;
+                            type = T_P2_CAND; a = pc; b = pq >> 16; ng = (cnt + 15) >> 4;
+                            break;
+                        }
                         {
                             const int q = (myq + qoff) & 3;
                             if (P.n_cu > 0 && !((cand_exh >> q) & 1) && ndefer < NDEFER && (ctrl->sel_final || ctrl->sel_ready)) {
