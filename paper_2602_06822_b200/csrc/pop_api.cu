@@ -60,19 +60,20 @@ static int check_shape(int d, int N, pop_dtype_t dt) {
     return POP_OK;
 }
 
-template <typename P>
-static int dev_alloc(P** ptr, size_t bytes) {
-    *ptr = nullptr;
-    if (bytes == 0) bytes = 16;
-    POP_CUDA(cudaMalloc((void**)ptr, bytes));
-    return POP_OK;
-}
+// All device buffers of a partition are carved out of one allocation (one cudaMalloc and one cudaFree per
+// partition: the calls, not the bytes, are what a prefill pays for), each on a 256-byte boundary.
+struct SlabPlan {
+    size_t total = 0;
+    size_t take(size_t bytes) {
+        const size_t at = total;
+        total += ((bytes ? bytes : 16) + 255) & ~(size_t)255;
+        return at;
+    }
+};
 
 static void partition_free(pop_partition* p) {
     if (!p) return;
-    cudaFree(p->GU); cudaFree(p->WdT); cudaFree(p->idx_ret); cudaFree(p->idx_cand); cudaFree(p->idx_pruned);
-    cudaFree(p->scores); cudaFree(p->norm_cand); cudaFree(p->h); cudaFree(p->keys); cudaFree(p->y_acc);
-    cudaFree(p->sel_slots); cudaFree(p->sync); cudaFree(p->wnorm_cand); cudaFree(p->rpart);
+    cudaFree(p->slab);
     free(p);
 }
 
@@ -80,7 +81,6 @@ static void partition_free(pop_partition* p) {
 static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, cudaStream_t st, pop_partition** out) {
     pop_partition* p = (pop_partition*)calloc(1, sizeof(pop_partition));
     if (!p) return POP_ERR_ALLOC;
-    int rc = POP_OK;
     cudaError_t e = cudaGetDevice(&p->device);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaGetDevice"); free(p); return POP_ERR_CUDA; }
     p->d = d; p->N = N; p->dtype = dt; p->es = dt == POP_F32 ? 4 : 2;
@@ -101,32 +101,43 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     p->n_ct = (n_cand + 7) / 8;
     p->n_ret_pad = 16 * p->n_cg;
     p->h_stride = p->layout == POP_LAYOUT_TILED ? p->n_ret_pad + ((n_cand + 15) / 16) * 16 : (p->n_rc > 0 ? p->n_rc : 1);
-#define TRY(x) do { rc = (x); if (rc != POP_OK) { partition_free(p); return rc; } } while (0)
-    if (p->layout == POP_LAYOUT_TILED) {
-        TRY(dev_alloc(&p->GU, ((size_t)(p->n_rt + p->n_ct) * 16 + (size_t)n_cand * 2) * row));
-        TRY(dev_alloc(&p->WdT, ((size_t)p->n_ret_pad + (size_t)n_cand) * row));
-    } else {
-        TRY(dev_alloc(&p->GU, (size_t)p->n_rc * 2 * row));
-        TRY(dev_alloc(&p->WdT, (size_t)p->n_rc * row));
+    SlabPlan plan;
+    const size_t o_GU = plan.take(p->layout == POP_LAYOUT_TILED ? ((size_t)(p->n_rt + p->n_ct) * 16 + (size_t)n_cand * 2) * row
+                                                                : (size_t)p->n_rc * 2 * row);
+    const size_t o_WdT = plan.take(p->layout == POP_LAYOUT_TILED ? ((size_t)p->n_ret_pad + (size_t)n_cand) * row
+                                                                 : (size_t)p->n_rc * row);
+    const size_t o_ret = plan.take(sizeof(int32_t) * (size_t)n_ret);
+    const size_t o_cand = plan.take(sizeof(int32_t) * (size_t)n_cand);
+    const size_t o_pruned = plan.take(sizeof(int32_t) * (size_t)p->n_pruned);
+    const size_t o_scores = plan.take(sizeof(double) * (size_t)N);
+    const size_t o_norm = plan.take(sizeof(double) * (size_t)n_cand);
+    // (tiled layout: 8 bytes per element of h, the value with the epoch of the step that wrote it)
+    const size_t h_bytes = 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1);
+    const size_t o_h = plan.take(h_bytes);
+    const size_t o_keys = plan.take(sizeof(u64) * (size_t)n_cand);
+    const size_t o_yacc = plan.take(sizeof(float) * (size_t)POP_MAX_BATCH * d);
+    const size_t o_sel = plan.take(sizeof(int32_t) * (size_t)n_cand);
+    const size_t o_sync = plan.take(sizeof(u32) * SYNC_WORDS);
+    const size_t o_wnorm = plan.take(sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1));
+    const size_t o_rpart = plan.take(sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1));
+    e = cudaMalloc(&p->slab, plan.total);
+    if (e != cudaSuccess) {
+        pop_set_cuda_error(e, "cudaMalloc");
+        p->slab = nullptr;
+        partition_free(p);
+        return e == cudaErrorMemoryAllocation ? POP_ERR_ALLOC : POP_ERR_CUDA;
     }
-    TRY(dev_alloc(&p->idx_ret, sizeof(int32_t) * (size_t)n_ret));
-    TRY(dev_alloc(&p->idx_cand, sizeof(int32_t) * (size_t)n_cand));
-    TRY(dev_alloc(&p->idx_pruned, sizeof(int32_t) * (size_t)p->n_pruned));
-    TRY(dev_alloc(&p->scores, sizeof(double) * (size_t)N));
-    TRY(dev_alloc(&p->norm_cand, sizeof(double) * (size_t)n_cand));
-    // (tiled layout: 8 bytes per element, the value with the epoch of the step that wrote it)
-    TRY(dev_alloc(&p->h, 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1)));
-    TRY(dev_alloc(&p->keys, sizeof(u64) * (size_t)n_cand));
-    TRY(dev_alloc(&p->y_acc, sizeof(float) * (size_t)POP_MAX_BATCH * d));
-    TRY(dev_alloc(&p->sel_slots, sizeof(int32_t) * (size_t)n_cand));
-    TRY(dev_alloc(&p->sync, sizeof(u32) * SYNC_WORDS));
-    TRY(dev_alloc(&p->wnorm_cand, sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1)));
-    TRY(dev_alloc(&p->rpart, sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1)));
-#undef TRY
+    unsigned char* base = (unsigned char*)p->slab;
+    p->GU = base + o_GU; p->WdT = base + o_WdT;
+    p->idx_ret = (int32_t*)(base + o_ret); p->idx_cand = (int32_t*)(base + o_cand); p->idx_pruned = (int32_t*)(base + o_pruned);
+    p->scores = (double*)(base + o_scores); p->norm_cand = (double*)(base + o_norm);
+    p->h = (float*)(base + o_h); p->keys = (u64*)(base + o_keys); p->y_acc = (float*)(base + o_yacc);
+    p->sel_slots = (int32_t*)(base + o_sel); p->sync = (u32*)(base + o_sync);
+    p->wnorm_cand = (float*)(base + o_wnorm); p->rpart = (double*)(base + o_rpart);
     e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->scores, 0, sizeof(double) * (size_t)N, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1), st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, h_bytes, st);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free(p); return POP_ERR_CUDA; }
     *out = p;
     return POP_OK;

@@ -140,7 +140,8 @@ int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, con
 //
 // Block = 256 threads = 8 warps; block tile = 256 tokens x 32 channels (gate and up at once);
 // a warp owns 32 tokens x 32 channels, lane (tg, cg) = (lane / 8, lane % 8) a tile of 8 tokens x
-// 4 channels x {gate, up} = 64 accumulators.  K is consumed in chunks of 16, staged in shared
+// 4 channels x {gate, up} = 64 accumulators (channels 2 cg, 2 cg + 1, 16 + 2 cg, 17 + 2 cg, so that the
+// 16-byte loads of the 8 lanes that are served together cover 128 contiguous bytes: no bank conflict).  K is consumed in chunks of 16, staged in shared
 // memory as doubles ([k][token] and [k][channel], so a lane reads its operands as contiguous
 // 16-byte pieces that the lanes of a warp share by broadcast), double-buffered with the next
 // chunk's global loads in flight during the arithmetic.  blockIdx.y splits the tokens into
@@ -226,8 +227,8 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
             const int buf = kc & 1;
             if (kc + 1 < nk) fetch(kc + 1);
             const double* xs = Xs + (size_t)buf * G2_KT * G2_TOK + warp * 32 + tg * 8;
-            const double* gs = Gs + (size_t)buf * G2_KT * G2_CH + cg * 4;
-            const double* us = Us + (size_t)buf * G2_KT * G2_CH + cg * 4;
+            const double* gs = Gs + (size_t)buf * G2_KT * G2_CH + cg * 2;
+            const double* us = Us + (size_t)buf * G2_KT * G2_CH + cg * 2;
 #pragma unroll
             for (int k = 0; k < G2_KT; ++k) {
                 double xv[8], gv[4], uv[4];
@@ -237,9 +238,9 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
                     xv[j] = t2.x; xv[j + 1] = t2.y;
                 }
 #pragma unroll
-                for (int c = 0; c < 4; c += 2) {
-                    const double2 a2 = *reinterpret_cast<const double2*>(gs + k * G2_CH + c);
-                    const double2 b2 = *reinterpret_cast<const double2*>(us + k * G2_CH + c);
+                for (int c = 0; c < 4; c += 2) {        // channels 2 cg, 2 cg + 1, then 16 + 2 cg, 17 + 2 cg
+                    const double2 a2 = *reinterpret_cast<const double2*>(gs + k * G2_CH + c * 8);
+                    const double2 b2 = *reinterpret_cast<const double2*>(us + k * G2_CH + c * 8);
                     gv[c] = a2.x; gv[c + 1] = a2.y; uv[c] = b2.x; uv[c + 1] = b2.y;
                 }
 #pragma unroll
@@ -270,7 +271,7 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
     }
     if (tg == 0) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) red[warp][cg * 4 + c] = e[c];
+        for (int c = 0; c < 4; ++c) red[warp][(c >> 1) * 16 + cg * 2 + (c & 1)] = e[c];
     }
     __syncthreads();
     if (tid < G2_CH && chan[tid] >= 0) {
