@@ -310,6 +310,39 @@ def run_pop(args):
     e2e = timed(True, max(1, args.steps // 2), 1)
     e2e_steps = max(1, args.steps // 2)
 
+    def timed_variant(label, ratios_v, k_v, note):
+        """The method's two limiting variants (Table 5 / Sec. 4.6) through the same two calls, decode only:
+        one warm-up pass and two timed passes of `tokens` x `layers` layer-steps."""
+        nr, nc, npr, _ = pop.region_sizes(N, ratios_v)
+        parts = [pop.prefill_partition(X, *W[l], ratios_v) for l in range(layers)]
+        ms = []
+        for rep_i in range(3):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            ev[0].record(stream)
+            for t in range(tokens):
+                for l in range(layers):
+                    pop.decode_step(parts[l], xs[t], k_v, y=act[l + 1])
+            ev[1].record(stream)
+            torch.cuda.synchronize()
+            if rep_i:
+                ms.append(ev[0].elapsed_time(ev[1]))
+        for p_ in parts:
+            p_.check()
+        free(parts)
+        us = 1e3 * max_over_ranks(sum(ms) / len(ms), world, dev) / (layers * tokens)
+        vb = algorithmic_bytes_per_layer_step(d, es, nr, nc, k_v, B)
+        return {"variant": label, "n_ret": nr, "n_cand": nc, "k": k_v, "us_per_layer_step": us,
+                "algorithmic_bytes_per_launch": vb, "achieved_GBs": vb / (us * 1e-6) / 1e9, "note": note}
+
+    variants = []
+    if not args.no_variants:
+        n_act = n_ret + k
+        variants.append(timed_variant("static mask (Variant 1)", (n_act / N, 0.0, (N - n_act) / N), 0,
+                                      "mask fixed at prefill: the same active count, no candidate region, no per-step choice"))
+        variants.append(timed_variant("all channels candidates (Variant 2)", (0.0, 1.0, 0.0), n_act,
+                                      "every channel scored at every step; served by the fused kernel (the streaming kernel "
+                                      "holds up to 1536 candidates)"))
+
     def reduce_max(v):
         return max_over_ranks(v, world, dev)
 
@@ -357,6 +390,8 @@ def run_pop(args):
                          "frac_of_nominal_8TBs": achieved / 8000.0,
                          "kernel": "decode layer-step (all kernels of one pop_decode_step, averaged over the decode region)"},
         }
+        if variants:
+            line["variants"] = variants
         if cpu is not None:
             line["cpu_baseline"] = {k2: cpu[k2] for k2 in ("value", "unit", "cores", "kind", "sample")}
         print(json.dumps(line))
@@ -375,6 +410,7 @@ def main():
     ap.add_argument("--layers", type=int, default=8)
     ap.add_argument("--tokens", type=int, default=128)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the timing of the method's two limiting variants")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
