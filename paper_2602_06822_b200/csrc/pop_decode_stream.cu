@@ -354,14 +354,16 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, u
             kor |= __shfl_xor_sync(0xffffffffu, kor, off);
             kand &= __shfl_xor_sync(0xffffffffu, kand, off);
         }
+        POP_TRACE(19);
         // The k-th largest key up to its low bits: radix passes of 8 bits, skipping digits that all keys share,
-        // at most two counted passes (the bucket of keys that agree with the k-th largest on the digits looked
-        // at is far narrower than the error bounds anyway).
+        // at most two counted passes, and the second only while more than a few keys agree with the k-th largest on
+        // the digits looked at: every key of that bucket is re-scored exactly, so a bucket of a few keys costs
+        // nothing, and a counted pass costs this one warp 2.6 us.
         const u32 differ = kor ^ kand;
         u32 prefix = 0, mask = 0;
-        int rem = k, counted = 0;
+        int rem = k, counted = 0, bucket = n;
 #pragma unroll 1
-        for (int shift = 24; shift >= 0 && counted < 2; shift -= 8) {
+        for (int shift = 24; shift >= 0 && counted < 2 && bucket > 24; shift -= 8) {
             if (((differ >> shift) & 255u) == 0u) {
                 prefix |= kor & (255u << shift);
                 mask |= 255u << shift;
@@ -386,18 +388,19 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, u
                 if (lane + off < 32) incl += t;
             }
             const u32 above = incl - tot;
-            u32 found = 0xffffffffu, cumf = 0;
+            u32 found = 0xffffffffu, cumf = 0, cntf = 0;
             if (above < (u32)rem && (u32)rem <= above + tot) {
                 u32 cum = above;
 #pragma unroll
                 for (int j = 7; j >= 0; --j) {
-                    if (found == 0xffffffffu && cum + c[j] >= (u32)rem) { found = 8 * lane + j; cumf = cum; }
+                    if (found == 0xffffffffu && cum + c[j] >= (u32)rem) { found = 8 * lane + j; cumf = cum; cntf = c[j]; }
                     cum += c[j];
                 }
             }
             const int src = __ffs(__ballot_sync(0xffffffffu, found != 0xffffffffu)) - 1;
             found = __shfl_sync(0xffffffffu, found, src);
             cumf = __shfl_sync(0xffffffffu, cumf, src);
+            bucket = (int)__shfl_sync(0xffffffffu, cntf, src);
             rem -= (int)cumf;
             prefix |= found << shift;
             mask |= 255u << shift;
@@ -405,6 +408,7 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, u
             __syncwarp();
         }
         // fewer than k keys lie above the bucket [prefix, prefix | ~mask], at least k at or above its lower end
+        POP_TRACE(20);
         // thresholds as key bit patterns, rounded away from the bucket (keys are non-negative floats: they order
         // like their bit patterns)
         const double m2 = 2.0 * (double)mm;
