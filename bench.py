@@ -169,9 +169,9 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- measured DRAM traffic
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu capture summarised in
-# profiles/pop_decode_stream_kernel_llama2_7b_r20_b1.md (226.07 MB read + 9.5 MB written).  Valid for the default
-# decode kernel of that workload only; None for anything else, and to be reset to None when that kernel changes.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from an ncu capture of the streaming
+# kernel on this workload (226.07 MB read + 9.5 MB written; the summary is kept with the profiles).  Valid for the
+# default decode kernel of that workload only; None for anything else, and to be reset to None when that kernel changes.
 NCU_TRAFFIC_BYTES = {"llama2_7b_ffn_r20_b1": 235.6e6}
 
 

@@ -3,7 +3,7 @@
 Comparison rules (stated here once, used by every parity test):
   * index sets (regions, selected candidates) must be equal arrays, except that ids may swap
     across a rank boundary when their ORACLE scores lie within 1e-6 relative of the oracle's
-    score at that boundary (north-star allowance for near-ties);
+    score at that boundary (allowance for near-ties: such scores are equal for every practical purpose);
   * outputs: err_j = |y_j - yref_j| / max(|yref_j|, 1e-2 * max_j |yref_j|); max_j err_j must be
     <= 1e-4 for fp32 and <= 2e-2 for bf16.  The floor keeps the measure meaningful for outputs
     that happen to lie near zero, where an fp32 accumulation has an absolute, not a relative,
