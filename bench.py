@@ -109,7 +109,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- oracle leg (CPU)
-def oracle_sample(name, seed=0, prompt_sample=64, decode_sample=4):
+def oracle_sample(name, seed=0, prompt_sample=64, decode_sample=4, one_thread=False):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload: the prefill
     partition from the first `prompt_sample` prompt tokens and `decode_sample` decode steps."""
     from oracle import pop_oracle as po
@@ -135,10 +135,23 @@ def oracle_sample(name, seed=0, prompt_sample=64, decode_sample=4):
         po.decode_step(xs[t], *Wh, part["R"], part["C"], k)
     t2 = time.perf_counter()
     per_step = (t2 - t1) / decode_sample
-    return {"value": 1.0 / per_step, "unit": "layer-steps/s", "cores": int(threads), "kind": "oracle",
-            "sample": f"1 layer: prefill partition on {X.shape[0]} of {L * B} prompt tokens ({t1 - t0:.2f} s), "
-                      f"then {decode_sample} decode layer-steps ({per_step * 1e3:.1f} ms each)",
-            "prefill_s": t1 - t0, "decode_s_per_layer_step": per_step}
+    out = {"value": 1.0 / per_step, "unit": "layer-steps/s", "cores": int(threads), "kind": "oracle",
+           "sample": f"1 layer: prefill partition on {X.shape[0]} of {L * B} prompt tokens ({t1 - t0:.2f} s), "
+                     f"then {decode_sample} decode layer-steps ({per_step * 1e3:.1f} ms each)",
+           "prefill_s": t1 - t0, "decode_s_per_layer_step": per_step}
+    if one_thread:
+        # the same decode step with the numerical library held to one thread
+        try:
+            from threadpoolctl import threadpool_limits
+            with threadpool_limits(limits=1):
+                t3 = time.perf_counter()
+                po.decode_step(xs[0], *Wh, part["R"], part["C"], k)
+                t4 = time.perf_counter()
+            out["value_one_thread"] = 1.0 / (t4 - t3)
+            out["sample"] += f"; one more step on 1 thread ({(t4 - t3) * 1e3:.0f} ms)"
+        except ImportError:
+            pass
+    return out
 
 
 def run_reference(args):
@@ -364,7 +377,7 @@ def run_pop(args):
         peak_src = "measured (MEASURED_PEAKS.json hbm_gbs)" if "hbm_gbs" in peaks else "fallback 6650 GB/s"
         abytes = algorithmic_bytes_per_layer_step(d, es, n_ret, n_cand, k, B)
         achieved = abytes / (us_per_ls * 1e-6) / 1e9
-        cpu = oracle_sample(name) if world == 1 and not args.no_cpu_baseline else None
+        cpu = oracle_sample(name, one_thread=True) if world == 1 and not args.no_cpu_baseline else None
         line = {
             "metric": "pop_decode_layer_steps_per_s", "value": value, "unit": "layer-steps/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_ms / args.steps,
@@ -393,7 +406,7 @@ def run_pop(args):
         if variants:
             line["variants"] = variants
         if cpu is not None:
-            line["cpu_baseline"] = {k2: cpu[k2] for k2 in ("value", "unit", "cores", "kind", "sample")}
+            line["cpu_baseline"] = {k2: cpu[k2] for k2 in ("value", "unit", "cores", "kind", "sample", "value_one_thread") if k2 in cpu}
         print(json.dumps(line))
     if world > 1:
         dist.barrier()
