@@ -169,11 +169,16 @@ def run_reference(args):
     per = statistics.mean(v["decode_s_per_layer_step"] for v in vals)
     total = sum(v["decode_s_per_layer_step"] * 2 + v["prefill_s"] for v in vals)
     d, N, dt, L, B, r = WORKLOADS[name]
+    from oracle import pop_oracle as po
+    nr, nc, _np = po.region_sizes(N, ratios_of(name))
+    kd = nc // 2
     value = 1.0 / per
     line = {"impl": "reference", "metric": "pop_decode_layer_steps_per_s", "value": value, "unit": "layer-steps/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": name, "d": d, "N": N, "batch": B, "ratios": list(ratios_of(name))},
+            "config": {"workload": name, "d": d, "N": N, "batch": B, "prompt_tokens": L * B, "ratios": list(ratios_of(name)),
+                       "n_ret": int(nr), "n_cand": int(nc), "k": int(kd), "layers": args.layers, "tokens": args.tokens,
+                       "sample_per_step": "one layer: prefill partition on 32 prompt tokens + 2 decode layer-steps"},
             "cpu_baseline": {"value": value, "unit": "layer-steps/s", "cores": vals[-1]["cores"], "kind": "oracle",
                              "sample": "per step: prefill partition on 32 prompt tokens + 2 decode layer-steps of one layer"},
             "e2e": {"value": value, "unit": "layer-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
