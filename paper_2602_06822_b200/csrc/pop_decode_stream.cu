@@ -1172,6 +1172,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
 #ifdef POP_STREAM_TRACE
             if (w == 0 && cd.x == T_P2_RET && cq < 0) POP_TRACE(11);
             if (w == 0 && cd.x == T_P2_CAND && !g_trace[cta * TRACE_SLOTS + 12]) POP_TRACE(12);
+            if (w == 0 && lane == 0) {
+                g_trace[cta * TRACE_SLOTS + 21] = (unsigned long long)cd.x;                       // type of the last unit
+                g_trace[cta * TRACE_SLOTS + (cd.x == T_P2_CAND ? 22 : 23)] += (unsigned long long)cd.w;   // groups by type
+                g_trace[cta * TRACE_SLOTS + 24] = trace_now();                                    // start of the last unit
+            }
 #endif
 
             // ---- unit prologue
