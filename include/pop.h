@@ -144,12 +144,22 @@ int pop_partition_destroy(pop_partition_t* p);
  *   h[b, i] = silu(Wg[i].x[b]) * (Wu[i].x[b]) for i in R u C;
  *   score_i = ||Wd[:, i]||_2 * sqrt(sum_b h[b, i]^2) for i in C (one mask shared by the batch);
  *   M = the k_candidate candidates with the largest (score descending, channel id ascending),
- *       decided on fp64 scores;
+ *       as exact (fp64) scores rank them: kernels that score in lower precision keep a bound of
+ *       each score's error and re-score in fp64 every candidate the bounds cannot separate from
+ *       the k-th;
  *   y[b] = sum over i in R u M of Wd[:, i] * h[b, i]   (fp32 accumulation).
  *   mask_out: uint8 [n_cand], 1 where the candidate in that slot (slot order = the d_cand array)
  *             was selected; may be NULL.
  *   sel_out : int32 [k_candidate], channel ids of the selected candidates, ascending; may be NULL.
  * No allocation, no host synchronisation.  0 <= k_candidate <= n_cand.
+ * One partition serves one stream at a time (its scratch and counters are shared by its steps).
+ * Two steps of the same call sequence may differ in the last bit of y: partial sums are added to
+ * the fp32 accumulator in the order the SMs deliver them; the mask does not depend on that order.
+ * The default kernel for bf16 partitions with d in {2048, 4096, 5120} is launched so that its CTAs
+ * may take over SMs from the previous kernel of the stream; callers that keep other streams busy
+ * on the same device should set POP_STREAM_LAUNCH=coop (cooperative launch) before the first step:
+ * a step whose CTAs cannot all be resident ends with POP_ERR_TIMEOUT at the next
+ * pop_partition_check instead of hanging.
  * Errors: POP_ERR_INVALID_ARG, POP_ERR_UNSUPPORTED (B too large for the shape), POP_ERR_CUDA.
  */
 int pop_decode_step(pop_partition_t* p, const void* x, int B, int k_candidate,
