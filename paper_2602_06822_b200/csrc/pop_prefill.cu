@@ -2,6 +2,7 @@
 //   column norms of the down projection, per-channel activation energy over the prompt,
 //   importance scores, rank-select into Retained / Candidate / Pruned, weight repack.
 #include "pop_common.cuh"
+#include <stdlib.h>
 #include "pop_select.cuh"
 
 // ---------------------------------------------------------------------------------------------
@@ -141,7 +142,8 @@ int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, con
 // Block = 256 threads = 8 warps; block tile = 256 tokens x 32 channels (gate and up at once);
 // a warp owns 32 tokens x 32 channels, lane (tg, cg) = (lane / 8, lane % 8) a tile of 8 tokens x
 // 4 channels x {gate, up} = 64 accumulators (channels 2 cg, 2 cg + 1, 16 + 2 cg, 17 + 2 cg, so that the
-// 16-byte loads of the 8 lanes that are served together cover 128 contiguous bytes: no bank conflict).  K is consumed in chunks of 16, staged in shared
+// 16-byte loads of the 8 lanes that are served together cover 128 contiguous bytes: no bank conflict).
+// K is consumed in chunks of KT (16; 32 for bf16, which halves the block barriers), staged in shared
 // memory as doubles ([k][token] and [k][channel], so a lane reads its operands as contiguous
 // 16-byte pieces that the lanes of a warp share by broadcast), double-buffered with the next
 // chunk's global loads in flight during the arithmetic.  blockIdx.y splits the tokens into
@@ -152,17 +154,17 @@ int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, con
 #define G2_CH 32
 #define G2_KT 16
 
-template <typename T>
+template <typename T, int KT>
 __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
     const T* __restrict__ X, int L, int d, const T* __restrict__ Wg, const T* __restrict__ Wu,
     const int32_t* __restrict__ chan_list, int n_list, int tok_per_split, double* __restrict__ s2out, int out_stride) {
     constexpr int EPV = 16 / sizeof(T);               // elements per 16-byte vector
-    constexpr int XV = G2_KT / EPV;                   // vectors per token row and chunk
-    constexpr int WV = 8 / EPV;                       // vectors per (matrix, channel, half chunk)
+    constexpr int XV = KT / EPV;                   // vectors per token row and chunk
+    constexpr int WV = (KT / 2) / EPV;                // vectors per (matrix, channel, half chunk)
     extern __shared__ __align__(16) double g2_sm[];
-    double* Xs = g2_sm;                               // [2][G2_KT][G2_TOK]
-    double* Gs = Xs + 2 * G2_KT * G2_TOK;             // [2][G2_KT][G2_CH]
-    double* Us = Gs + 2 * G2_KT * G2_CH;
+    double* Xs = g2_sm;                               // [2][KT][G2_TOK]
+    double* Gs = Xs + 2 * KT * G2_TOK;             // [2][KT][G2_CH]
+    double* Us = Gs + 2 * KT * G2_CH;
     __shared__ int chan[G2_CH];
     __shared__ double red[8][G2_CH];
 
@@ -174,12 +176,12 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
     }
     __syncthreads();
     const int t_begin = blockIdx.y * tok_per_split, t_end = min(L, t_begin + tok_per_split);
-    const int nk = d / G2_KT;
+    const int nk = d / KT;
 
     // staging roles: every thread one token row of X; threads 0..127 one (matrix, channel, half chunk) of W
     const int wm = tid >> 6, wc = (tid >> 1) & 31, wh = tid & 1;
     const int wch = tid < 128 ? chan[wc] : -1;
-    const T* wrow = wch >= 0 ? (wm ? Wu : Wg) + (size_t)wch * d + wh * 8 : nullptr;
+    const T* wrow = wch >= 0 ? (wm ? Wu : Wg) + (size_t)wch * d + wh * (KT / 2) : nullptr;
 
     double e[4] = {0.0, 0.0, 0.0, 0.0};
     for (int t0 = t_begin; t0 < t_end; t0 += G2_TOK) {
@@ -189,10 +191,10 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
         auto fetch = [&](int kc) {
 #pragma unroll
             for (int v = 0; v < XV; ++v)
-                xr[v] = xrow ? __ldg(reinterpret_cast<const uint4*>(xrow + kc * G2_KT) + v) : make_uint4(0u, 0u, 0u, 0u);
+                xr[v] = xrow ? __ldg(reinterpret_cast<const uint4*>(xrow + kc * KT) + v) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
             for (int v = 0; v < WV; ++v)
-                wr[v] = wrow ? __ldg(reinterpret_cast<const uint4*>(wrow + kc * G2_KT) + v) : make_uint4(0u, 0u, 0u, 0u);
+                wr[v] = wrow ? __ldg(reinterpret_cast<const uint4*>(wrow + kc * KT) + v) : make_uint4(0u, 0u, 0u, 0u);
         };
         auto stash = [&](int buf) {
 #pragma unroll
@@ -200,7 +202,7 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
                 float f[EPV];
                 Elem<T>::unpack(xr[v], f);
 #pragma unroll
-                for (int j = 0; j < EPV; ++j) Xs[(buf * G2_KT + v * EPV + j) * G2_TOK + tid] = (double)f[j];
+                for (int j = 0; j < EPV; ++j) Xs[(buf * KT + v * EPV + j) * G2_TOK + tid] = (double)f[j];
             }
             if (tid < 128) {
                 double* dst = wm ? Us : Gs;
@@ -209,7 +211,7 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
                     float f[EPV];
                     Elem<T>::unpack(wr[v], f);
 #pragma unroll
-                    for (int j = 0; j < EPV; ++j) dst[(buf * G2_KT + wh * 8 + v * EPV + j) * G2_CH + wc] = (double)f[j];
+                    for (int j = 0; j < EPV; ++j) dst[(buf * KT + wh * (KT / 2) + v * EPV + j) * G2_CH + wc] = (double)f[j];
                 }
             }
         };
@@ -226,11 +228,11 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
         for (int kc = 0; kc < nk; ++kc) {
             const int buf = kc & 1;
             if (kc + 1 < nk) fetch(kc + 1);
-            const double* xs = Xs + (size_t)buf * G2_KT * G2_TOK + warp * 32 + tg * 8;
-            const double* gs = Gs + (size_t)buf * G2_KT * G2_CH + cg * 2;
-            const double* us = Us + (size_t)buf * G2_KT * G2_CH + cg * 2;
+            const double* xs = Xs + (size_t)buf * KT * G2_TOK + warp * 32 + tg * 8;
+            const double* gs = Gs + (size_t)buf * KT * G2_CH + cg * 2;
+            const double* us = Us + (size_t)buf * KT * G2_CH + cg * 2;
 #pragma unroll
-            for (int k = 0; k < G2_KT; ++k) {
+            for (int k = 0; k < KT; ++k) {
                 double xv[8], gv[4], uv[4];
 #pragma unroll
                 for (int j = 0; j < 8; j += 2) {
@@ -295,33 +297,33 @@ int pop_prefill_s2_gemm_splits(int L) { return L > 0 ? (L + G2_TOK - 1) / G2_TOK
 
 bool pop_prefill_s2_gemm_supported(int d) { return d >= G2_KT && d % G2_KT == 0; }
 
+template <typename T, int KT>
+static int launch_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, double* s2part, cudaStream_t st) {
+    auto kern = prefill_s2_gemm_kernel<T, KT>;
+    const size_t smem = sizeof(double) * (2 * KT * G2_TOK + 4 * KT * G2_CH);
+    static thread_local int cfg_dev = -1;
+    int dev = 0;
+    POP_CUDA(cudaGetDevice(&dev));
+    if (cfg_dev != dev) {
+        POP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        cfg_dev = dev;
+    }
+    dim3 grd((N + G2_CH - 1) / G2_CH, pop_prefill_s2_gemm_splits(L));
+    kern<<<grd, 256, smem, st>>>((const T*)X, L, d, (const T*)Wg, (const T*)Wu, nullptr, N, G2_TOK, s2part, N);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
 int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
                                double* s2part, double* s2, cudaStream_t st) {
     if (N <= 0) return POP_OK;
-    const int nsplit = pop_prefill_s2_gemm_splits(L);
-    const size_t smem = sizeof(double) * (2 * G2_KT * G2_TOK + 4 * G2_KT * G2_CH);
-    dim3 grd((N + G2_CH - 1) / G2_CH, nsplit);
-    static thread_local int cfg_dev[2] = {-1, -1};
-    int dev = 0;
-    POP_CUDA(cudaGetDevice(&dev));
-    if (dt == POP_F32) {
-        auto kern = prefill_s2_gemm_kernel<float>;
-        if (cfg_dev[0] != dev) {
-            POP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            cfg_dev[0] = dev;
-        }
-        kern<<<grd, 256, smem, st>>>((const float*)X, L, d, (const float*)Wg, (const float*)Wu, nullptr, N, G2_TOK, s2part, N);
-    } else {
-        auto kern = prefill_s2_gemm_kernel<__nv_bfloat16>;
-        if (cfg_dev[1] != dev) {
-            POP_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            cfg_dev[1] = dev;
-        }
-        kern<<<grd, 256, smem, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu,
-                                     nullptr, N, G2_TOK, s2part, N);
-    }
-    POP_LAUNCHED();
-    sum_ranges_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2part, nsplit, N, s2);
+    static const int kt_env = getenv("POP_PREFILL_KT") ? atoi(getenv("POP_PREFILL_KT")) : 32;
+    int rc;
+    if (dt == POP_F32) rc = launch_s2_gemm<float, G2_KT>(X, L, d, Wg, Wu, N, s2part, st);
+    else if (d % 32 == 0 && kt_env == 32) rc = launch_s2_gemm<__nv_bfloat16, 32>(X, L, d, Wg, Wu, N, s2part, st);
+    else rc = launch_s2_gemm<__nv_bfloat16, G2_KT>(X, L, d, Wg, Wu, N, s2part, st);
+    if (rc != POP_OK) return rc;
+    sum_ranges_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2part, pop_prefill_s2_gemm_splits(L), N, s2);
     POP_LAUNCHED();
     return POP_OK;
 }
