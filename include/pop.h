@@ -134,7 +134,12 @@ int pop_partition_shape(const pop_partition_t* p, int* d, int* N, pop_dtype_t* d
  */
 int pop_partition_check(pop_partition_t* p);
 
-/* Frees everything the partition owns.  The caller must have synchronised its stream. */
+/*
+ * Releases everything the partition owns.  The caller must have synchronised the work that used
+ * it.  Its device memory may stay with the library for the next partition of the same size on
+ * the same device (at most POP_SLAB_CACHE_MB megabytes in all, environment, default 4096, 0 = none):
+ * building a partition per prompt and layer then costs no cudaMalloc / cudaFree.
+ */
 int pop_partition_destroy(pop_partition_t* p);
 
 /*

@@ -4,6 +4,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
+#include <vector>
+
 #include "pop_common.cuh"
 
 static thread_local char g_cuda_err[256] = "";
@@ -71,9 +74,63 @@ struct SlabPlan {
     }
 };
 
+// Freed slabs are kept for the next partition of the same device and size instead of going back to the driver:
+// a serving loop builds one partition per prompt and layer, and cudaMalloc / cudaFree (which synchronises the
+// whole device) would otherwise sit in that path.  The cache holds at most POP_SLAB_CACHE_MB megabytes
+// (environment, read once; default 4096; 0 turns it off); what does not fit is freed at once.  A slab enters
+// the cache only through pop_partition_destroy, whose contract is that the caller has synchronised the work
+// that used it.
+namespace {
+struct CachedSlab { int device; size_t bytes; void* ptr; };
+std::mutex g_slab_mutex;
+std::vector<CachedSlab> g_slabs;
+size_t g_slab_bytes = 0;
+
+size_t slab_cache_limit() {
+    static const size_t limit = (size_t)(getenv("POP_SLAB_CACHE_MB") ? atoll(getenv("POP_SLAB_CACHE_MB")) : 4096) << 20;
+    return limit;
+}
+
+void* slab_take(int device, size_t bytes) {
+    std::lock_guard<std::mutex> lock(g_slab_mutex);
+    for (size_t i = 0; i < g_slabs.size(); ++i) {
+        if (g_slabs[i].device == device && g_slabs[i].bytes == bytes) {
+            void* ptr = g_slabs[i].ptr;
+            g_slab_bytes -= bytes;
+            g_slabs.erase(g_slabs.begin() + (long)i);
+            return ptr;
+        }
+    }
+    return nullptr;
+}
+
+void slab_flush() {                      // gives everything back to the driver (current device must own the slabs freed)
+    std::lock_guard<std::mutex> lock(g_slab_mutex);
+    int cur = 0;
+    cudaGetDevice(&cur);
+    for (size_t i = 0; i < g_slabs.size();) {
+        if (g_slabs[i].device == cur) {
+            cudaFree(g_slabs[i].ptr);
+            g_slab_bytes -= g_slabs[i].bytes;
+            g_slabs.erase(g_slabs.begin() + (long)i);
+        } else {
+            ++i;
+        }
+    }
+}
+
+bool slab_keep(int device, size_t bytes, void* ptr) {
+    std::lock_guard<std::mutex> lock(g_slab_mutex);
+    if (g_slab_bytes + bytes > slab_cache_limit()) return false;
+    g_slabs.push_back(CachedSlab{device, bytes, ptr});
+    g_slab_bytes += bytes;
+    return true;
+}
+}  // namespace
+
 static void partition_free(pop_partition* p) {
     if (!p) return;
-    cudaFree(p->slab);
+    if (p->slab && !slab_keep(p->device, p->slab_bytes, p->slab)) cudaFree(p->slab);
     free(p);
 }
 
@@ -120,7 +177,14 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     const size_t o_sync = plan.take(sizeof(u32) * SYNC_WORDS);
     const size_t o_wnorm = plan.take(sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1));
     const size_t o_rpart = plan.take(sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1));
-    e = cudaMalloc(&p->slab, plan.total);
+    p->slab_bytes = plan.total;
+    p->slab = slab_take(p->device, plan.total);
+    e = p->slab ? cudaSuccess : cudaMalloc(&p->slab, plan.total);
+    if (e == cudaErrorMemoryAllocation) {          // out of memory with slabs in the cache: give them back and try again
+        (void)cudaGetLastError();
+        slab_flush();
+        e = cudaMalloc(&p->slab, plan.total);
+    }
     if (e != cudaSuccess) {
         pop_set_cuda_error(e, "cudaMalloc");
         p->slab = nullptr;

@@ -48,6 +48,7 @@ struct pop_partition {
     int n_rt, n_ct, n_cg, n_ret_pad, h_stride;      // tiled layout only (h_stride: both)
 
     void* slab;                   // the one device allocation all pointers below point into
+    size_t slab_bytes;
     void* GU;
     void* WdT;
     int32_t* idx_ret;
