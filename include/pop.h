@@ -79,8 +79,10 @@ int pop_region_sizes(int N, pop_ratios_t ratios, int* n_ret, int* n_cand, int* n
  *   ranks channels by (I_i descending, i ascending): the first n_ret are Retained, the next
  *   n_cand Candidate, the rest Pruned (sizes as pop_region_sizes);
  *   repacks Wg/Wu rows and Wd columns of Retained then Candidate channels contiguously.
- * The ranking is decided on fp64 scores.  *out receives a new partition (destroy it with
- * pop_partition_destroy).  Allocates device memory (about (n_ret + n_cand) * 3 * d elements).
+ * The ranking is the one exact (fp64) scores give: see pop_partition_scores.  For bf16 the dense
+ * contraction runs on the tensor cores (tcgen05, operands through TMA) when d >= 64.
+ * *out receives a new partition (destroy it with pop_partition_destroy).  Allocates device memory
+ * (about (n_ret + n_cand) * 3 * d elements, plus stream-ordered temporaries).
  * Requirements: d * sizeof(element) a multiple of 16; pointers 16-byte aligned; L >= 1.
  * Errors: POP_ERR_INVALID_ARG, POP_ERR_UNSUPPORTED, POP_ERR_ALLOC, POP_ERR_CUDA.
  */
@@ -111,8 +113,18 @@ int pop_partition_sizes(const pop_partition_t* p, int* n_ret, int* n_cand, int* 
 int pop_partition_indices(const pop_partition_t* p, const int32_t** d_ret,
                           const int32_t** d_cand, const int32_t** d_pruned);
 
-/* Prefill importance scores I_i (Eq. 3), DEVICE double [N], owned by the partition. */
+/*
+ * Prefill importance scores I_i (Eq. 3), DEVICE double [N], owned by the partition, and a bound of
+ * the error of each, DEVICE double [N]: |scores[i] - I_i of exact arithmetic| <= bounds[i].
+ * fp32 partitions are scored in fp64 throughout (all bounds 0, scores within rounding of fp64).
+ * bf16 partitions are scored on the tensor cores (fp32 accumulation); every channel whose bound
+ * reaches one of the two rank boundaries (Retained | Candidate, Candidate | Pruned) is scored again
+ * in fp64 and carries that score with bound 0, so the regions are the ones exact scores give, while
+ * the scores of channels far from both boundaries are good to about 1e-4 relative.
+ * A partition built by pop_partition_from_indices has all scores and bounds 0.
+ */
 int pop_partition_scores(const pop_partition_t* p, const double** d_scores);
+int pop_partition_score_bounds(const pop_partition_t* p, const double** d_bounds);
 
 /*
  * Diagnostic view of the last decode step's candidate scoring (Sec. 3.3 decoding stage) on a
@@ -178,10 +190,14 @@ int pop_decode_step(pop_partition_t* p, const void* x, int B, int k_candidate,
  * inside a memory pool whose budget is fixed up front, a serving loop that forbids allocator
  * calls on its hot path because they may synchronise the device, or a host whose allocator
  * is owned by another framework.  pop_prefill_partition is closed to them, since it allocates the
- * partition and two stream-ordered temporaries.  This call computes the same I_i (Eq. 3; the
- * same kernels and the same fp64 arithmetic as pop_prefill_partition) into a buffer the caller
- * already owns, and keeps its temporaries (2 x N doubles) in a fixed 512 KB array that is part
- * of the library image on every GPU that loads it.
+ * partition and stream-ordered temporaries.  This call computes the same I_i (Eq. 3) into a buffer
+ * the caller already owns, and keeps its temporaries (2 x N doubles) in a fixed 512 KB array that is
+ * part of the library image on every GPU that loads it.  It scores every channel in fp64 with the
+ * library's plain per-channel kernel, not with the tensor-core pass or the blocked fp64 pass that
+ * pop_prefill_partition uses: the results agree with that call's scores to fp64 rounding where it
+ * reports an error bound of 0 and within its reported bound elsewhere (pop_partition_score_bounds), so
+ * a caller that ranks these scores gets the same regions up to ties at the last bit; it is also several
+ * times slower per layer (about 14 ms at hidden 4096, intermediate 11008, 512 prompt tokens).
  *   X [L, d], Wg [N, d], Wu [N, d], Wd [d, N]: device arrays of `dtype` as for
  *   pop_prefill_partition; scores_out: device double [N], caller-owned, written on `cuda_stream`.
  * It calls no cudaMalloc / cudaFree and no allocating library routine.

@@ -134,6 +134,15 @@ static void partition_free(pop_partition* p) {
     free(p);
 }
 
+// Error paths: work of this call may still be queued on the stream, so the slab goes straight back to the driver
+// (after the stream has drained) and never into the cache.
+static void partition_free_now(pop_partition* p, cudaStream_t st) {
+    if (!p) return;
+    cudaStreamSynchronize(st);
+    if (p->slab) cudaFree(p->slab);
+    free(p);
+}
+
 // Allocates the partition's buffers for given region sizes (contents undefined except zeroed scratch).
 static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, cudaStream_t st, pop_partition** out) {
     pop_partition* p = (pop_partition*)calloc(1, sizeof(pop_partition));
@@ -167,6 +176,7 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     const size_t o_cand = plan.take(sizeof(int32_t) * (size_t)n_cand);
     const size_t o_pruned = plan.take(sizeof(int32_t) * (size_t)p->n_pruned);
     const size_t o_scores = plan.take(sizeof(double) * (size_t)N);
+    const size_t o_bounds = plan.take(sizeof(double) * (size_t)N);
     const size_t o_norm = plan.take(sizeof(double) * (size_t)n_cand);
     // (tiled layout: 8 bytes per element of h, the value with the epoch of the step that wrote it)
     const size_t h_bytes = 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1);
@@ -187,22 +197,22 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     }
     if (e != cudaSuccess) {
         pop_set_cuda_error(e, "cudaMalloc");
-        p->slab = nullptr;
-        partition_free(p);
+        free(p);
         return e == cudaErrorMemoryAllocation ? POP_ERR_ALLOC : POP_ERR_CUDA;
     }
     unsigned char* base = (unsigned char*)p->slab;
     p->GU = base + o_GU; p->WdT = base + o_WdT;
     p->idx_ret = (int32_t*)(base + o_ret); p->idx_cand = (int32_t*)(base + o_cand); p->idx_pruned = (int32_t*)(base + o_pruned);
-    p->scores = (double*)(base + o_scores); p->norm_cand = (double*)(base + o_norm);
+    p->scores = (double*)(base + o_scores); p->score_bounds = (double*)(base + o_bounds); p->norm_cand = (double*)(base + o_norm);
     p->h = (float*)(base + o_h); p->keys = (u64*)(base + o_keys); p->y_acc = (float*)(base + o_yacc);
     p->sel_slots = (int32_t*)(base + o_sel); p->sync = (u32*)(base + o_sync);
     p->wnorm_cand = (float*)(base + o_wnorm); p->rpart = (double*)(base + o_rpart);
     e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->scores, 0, sizeof(double) * (size_t)N, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(p->score_bounds, 0, sizeof(double) * (size_t)N, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, h_bytes, st);
-    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free(p); return POP_ERR_CUDA; }
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free_now(p, st); return POP_ERR_CUDA; }
     *out = p;
     return POP_OK;
 }
@@ -225,31 +235,58 @@ extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg
     rc = partition_alloc(d, N, dtype, n_ret, n_cand, st, &p);
     if (rc != POP_OK) return rc;
 
-    // temporaries: column norms and activation energies, freed in stream order
-    double *norm = nullptr, *s2 = nullptr, *s2part = nullptr;
+    // temporaries (one stream-ordered allocation, freed in stream order): column norms, activation energies and,
+    // for the tensor-core pass, its partial sums, bounds and the re-scoring list
+    const bool tc = pop_prefill_tc_supported(d, dtype);
     const bool gemm = pop_prefill_s2_gemm_supported(d);
-    cudaError_t e = cudaMallocAsync((void**)&norm, sizeof(double) * (size_t)N, st);
-    if (e == cudaSuccess) e = cudaMallocAsync((void**)&s2, sizeof(double) * (size_t)N, st);
-    if (e == cudaSuccess && gemm)
-        e = cudaMallocAsync((void**)&s2part, sizeof(double) * (size_t)N * (size_t)pop_prefill_s2_gemm_splits(L), st);
+    PrefillTcPlan tp;
+    pop_prefill_tc_plan(L, d, N, &tp);
+    SlabPlan tmp;
+    const size_t t_norm = tmp.take(sizeof(double) * (size_t)N);
+    const size_t t_s2 = tmp.take(sizeof(double) * (size_t)N);
+    const size_t t_s2part = tmp.take(gemm ? sizeof(double) * (size_t)N * (size_t)pop_prefill_s2_gemm_splits(L) : 0);
+    size_t t_xn = 0, t_gn = 0, t_un = 0, t_tp = 0, t_bp = 0, t_mm = 0, t_list = 0, t_nl = 0, t_part = 0;
+    if (tc) {
+        t_xn = tmp.take(sizeof(float) * (size_t)tp.l_pad);
+        t_gn = tmp.take(sizeof(float) * (size_t)tp.n_pad);
+        t_un = tmp.take(sizeof(float) * (size_t)tp.n_pad);
+        t_tp = tmp.take(sizeof(double) * (size_t)tp.n_parts * tp.n_pad);
+        t_bp = tmp.take(sizeof(float) * (size_t)tp.n_parts * tp.n_pad);
+        t_mm = tmp.take(sizeof(u64));
+        t_list = tmp.take(sizeof(int32_t) * (size_t)N);
+        t_nl = tmp.take(sizeof(int));
+        t_part = tmp.take(sizeof(double) * (size_t)tp.max_list * tp.n_tb);
+    }
+    unsigned char* tb = nullptr;
+    cudaError_t e = cudaMallocAsync((void**)&tb, tmp.total, st);
     if (e != cudaSuccess) {
         pop_set_cuda_error(e, "cudaMallocAsync");
-        if (norm) cudaFreeAsync(norm, st);
-        if (s2) cudaFreeAsync(s2, st);
-        partition_free(p);
+        partition_free_now(p, st);
         return POP_ERR_ALLOC;
     }
+    double* norm = (double*)(tb + t_norm);
+    double* s2 = (double*)(tb + t_s2);
+    double* s2part = (double*)(tb + t_s2part);
     rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
-    if (rc == POP_OK) rc = gemm ? pop_launch_prefill_s2_gemm(X, L, d, Wg, Wu, N, dtype, s2part, s2, st)
-                                : pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
-    if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, p->scores, st);
+    if (rc == POP_OK && tc) {
+        PrefillTcScratch sc;
+        sc.xnorm = (float*)(tb + t_xn); sc.gnorm = (float*)(tb + t_gn); sc.unorm = (float*)(tb + t_un);
+        sc.s2part = (double*)(tb + t_tp); sc.bpart = (float*)(tb + t_bp); sc.m_max = (u64*)(tb + t_mm);
+        sc.list = (int32_t*)(tb + t_list); sc.n_list = (int*)(tb + t_nl); sc.part = (double*)(tb + t_part);
+        sc.s2part_full = s2part; sc.s2_full = s2;
+        rc = pop_launch_prefill_tc(X, L, d, Wg, Wu, N, norm, sc, p->scores, p->score_bounds, p->sync + SYNC_ERROR, p->sm_count, st);
+        if (rc == POP_OK)
+            rc = pop_launch_prefill_rescore(X, L, d, Wg, Wu, N, norm, n_ret, n_cand, sc, p->scores, p->score_bounds, p->sm_count, st);
+    } else if (rc == POP_OK) {
+        rc = gemm ? pop_launch_prefill_s2_gemm(X, L, d, Wg, Wu, N, dtype, s2part, s2, st)
+                  : pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
+        if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, p->scores, st);
+    }
     if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->idx_ret, p->idx_cand, p->idx_pruned, st);
     if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
                                                          : pop_launch_repack(p, Wg, Wu, Wd, norm, st);
-    cudaFreeAsync(norm, st);
-    cudaFreeAsync(s2, st);
-    if (s2part) cudaFreeAsync(s2part, st);
-    if (rc != POP_OK) { cudaStreamSynchronize(st); partition_free(p); return rc; }
+    cudaFreeAsync(tb, st);
+    if (rc != POP_OK) { partition_free_now(p, st); return rc; }
     *out = p;
     return POP_OK;
 }
@@ -298,15 +335,15 @@ extern "C" int pop_partition_from_indices(const void* Wg, const void* Wu, const 
     // the host arrays are pageable: wait so that the caller (and h_pruned) may go away
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     free(h_pruned);
-    if (e != cudaSuccess) { pop_set_cuda_error(e, "index upload"); partition_free(p); return POP_ERR_CUDA; }
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "index upload"); partition_free_now(p, st); return POP_ERR_CUDA; }
     double* norm = nullptr;
     e = cudaMallocAsync((void**)&norm, sizeof(double) * (size_t)N, st);
-    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMallocAsync"); partition_free(p); return POP_ERR_ALLOC; }
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMallocAsync"); partition_free_now(p, st); return POP_ERR_ALLOC; }
     rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
     if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
                                                          : pop_launch_repack(p, Wg, Wu, Wd, norm, st);
     cudaFreeAsync(norm, st);
-    if (rc != POP_OK) { cudaStreamSynchronize(st); partition_free(p); return rc; }
+    if (rc != POP_OK) { partition_free_now(p, st); return rc; }
     *out = p;
     return POP_OK;
 }
@@ -331,6 +368,12 @@ extern "C" int pop_partition_indices(const pop_partition_t* p, const int32_t** d
 extern "C" int pop_partition_scores(const pop_partition_t* p, const double** d_scores) {
     if (!p || !d_scores) return POP_ERR_INVALID_ARG;
     *d_scores = p->scores;
+    return POP_OK;
+}
+
+extern "C" int pop_partition_score_bounds(const pop_partition_t* p, const double** d_bounds) {
+    if (!p || !d_bounds) return POP_ERR_INVALID_ARG;
+    *d_bounds = p->score_bounds;
     return POP_OK;
 }
 

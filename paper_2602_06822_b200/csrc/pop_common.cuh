@@ -55,6 +55,7 @@ struct pop_partition {
     int32_t* idx_cand;
     int32_t* idx_pruned;
     double* scores;               // [N] prefill I_i
+    double* score_bounds;         // [N] bound of |scores[i] - exact I_i| (0 where the score is exact)
     double* norm_cand;            // [n_cand] ||Wd[:, i]||_2 of the candidate channels
     float* wnorm_cand;            // [2][n_cand] max |Wg[i][:]|, max |Wu[i][:]| of the candidate channels
     double* rpart;                // [4 n_cand][POP_MAX_BATCH] decode scratch: partial dot products of re-scoring jobs
@@ -114,6 +115,9 @@ bool pop_prefill_s2_gemm_supported(int d);
 int pop_prefill_s2_gemm_splits(int L);
 int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
                                double* s2part, double* s2, cudaStream_t st);
+// the same pass, enqueued always but run only when *run_if_gt > threshold (a device-side decision)
+int pop_launch_prefill_s2_gemm_if(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
+                                  double* s2part, double* s2, const int* run_if_gt, int threshold, cudaStream_t st);
 int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st);
 int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand,
                          int32_t* idx_ret, int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);
@@ -121,6 +125,31 @@ int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, co
                       const double* norm /*[N]*/, cudaStream_t st);
 int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                             const double* norm /*[N]*/, cudaStream_t st);
+// pop_prefill_tc.cu (bf16: activation energies on the tensor cores with error bounds, exact re-scoring of the
+// channels the bounds cannot place)
+#define POP_PREFILL_MAX_LIST 4096     // longest list the list re-scoring kernel takes; longer lists use the full fp64 pass
+struct PrefillTcPlan { int n_ct, n_tt, n_pad, l_pad, n_parts, n_tb, max_list; };
+struct PrefillTcScratch {
+    float* xnorm;          // [l_pad]
+    float* gnorm;          // [n_pad]
+    float* unorm;          // [n_pad]
+    double* s2part;        // [n_parts][n_pad]
+    float* bpart;          // [n_parts][n_pad]
+    u64* m_max;            // largest score bound (bits of a double)
+    int32_t* list;         // [N] channels to re-score
+    int* n_list;
+    double* part;          // [max_list][n_tb]
+    double* s2part_full;   // [pop_prefill_s2_gemm_splits(L)][N]
+    double* s2_full;       // [N]
+};
+bool pop_prefill_tc_supported(int d, pop_dtype_t dt);
+void pop_prefill_tc_plan(int L, int d, int N, PrefillTcPlan* plan);
+int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
+                          const PrefillTcScratch& s, double* scores, double* bounds, u32* status, int sm_count,
+                          cudaStream_t st);
+int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
+                               int n_ret, int n_cand, const PrefillTcScratch& s, double* scores, double* bounds,
+                               int sm_count, cudaStream_t st);
 // pop_decode_stream.cu (bf16 partitions in the tiled layout)
 bool pop_stream_layout_supported(int d, pop_dtype_t dt);
 int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void* y,

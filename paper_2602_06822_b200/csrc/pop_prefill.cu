@@ -157,7 +157,9 @@ int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, con
 template <typename T, int KT>
 __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
     const T* __restrict__ X, int L, int d, const T* __restrict__ Wg, const T* __restrict__ Wu,
-    const int32_t* __restrict__ chan_list, int n_list, int tok_per_split, double* __restrict__ s2out, int out_stride) {
+    const int32_t* __restrict__ chan_list, int n_list, int tok_per_split, double* __restrict__ s2out, int out_stride,
+    const int* __restrict__ run_if_gt, int threshold) {
+    if (run_if_gt && *run_if_gt <= threshold) return;           // the same decision in every thread of the grid
     constexpr int EPV = 16 / sizeof(T);               // elements per 16-byte vector
     constexpr int XV = KT / EPV;                   // vectors per token row and chunk
     constexpr int WV = (KT / 2) / EPV;                // vectors per (matrix, channel, half chunk)
@@ -285,9 +287,10 @@ __global__ void __launch_bounds__(256, 1) prefill_s2_gemm_kernel(
 }
 
 // s2[i] = sum over the token ranges (ascending) of s2part[y][i]
-__global__ void sum_ranges_kernel(const double* __restrict__ s2part, int nsplit, int N, double* __restrict__ s2) {
+__global__ void sum_ranges_kernel(const double* __restrict__ s2part, int nsplit, int N, double* __restrict__ s2,
+                                  const int* __restrict__ run_if_gt, int threshold) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N) return;
+    if (i >= N || (run_if_gt && *run_if_gt <= threshold)) return;
     double sum = 0.0;
     for (int y = 0; y < nsplit; ++y) sum += s2part[(size_t)y * N + i];
     s2[i] = sum;
@@ -298,7 +301,8 @@ int pop_prefill_s2_gemm_splits(int L) { return L > 0 ? (L + G2_TOK - 1) / G2_TOK
 bool pop_prefill_s2_gemm_supported(int d) { return d >= G2_KT && d % G2_KT == 0; }
 
 template <typename T, int KT>
-static int launch_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, double* s2part, cudaStream_t st) {
+static int launch_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, double* s2part,
+                          const int* run_if_gt, int threshold, cudaStream_t st) {
     auto kern = prefill_s2_gemm_kernel<T, KT>;
     const size_t smem = sizeof(double) * (2 * KT * G2_TOK + 4 * KT * G2_CH);
     static thread_local int cfg_dev = -1;
@@ -309,23 +313,28 @@ static int launch_s2_gemm(const void* X, int L, int d, const void* Wg, const voi
         cfg_dev = dev;
     }
     dim3 grd((N + G2_CH - 1) / G2_CH, pop_prefill_s2_gemm_splits(L));
-    kern<<<grd, 256, smem, st>>>((const T*)X, L, d, (const T*)Wg, (const T*)Wu, nullptr, N, G2_TOK, s2part, N);
+    kern<<<grd, 256, smem, st>>>((const T*)X, L, d, (const T*)Wg, (const T*)Wu, nullptr, N, G2_TOK, s2part, N, run_if_gt, threshold);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
+int pop_launch_prefill_s2_gemm_if(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
+                                  double* s2part, double* s2, const int* run_if_gt, int threshold, cudaStream_t st) {
+    if (N <= 0) return POP_OK;
+    int rc;
+    // K chunks of 32 for bf16 (half the block barriers of 16; measured 4.33 -> 4.14 ms at d 4096, N 11008, L 512)
+    if (dt == POP_F32) rc = launch_s2_gemm<float, G2_KT>(X, L, d, Wg, Wu, N, s2part, run_if_gt, threshold, st);
+    else if (d % 32 == 0) rc = launch_s2_gemm<__nv_bfloat16, 32>(X, L, d, Wg, Wu, N, s2part, run_if_gt, threshold, st);
+    else rc = launch_s2_gemm<__nv_bfloat16, G2_KT>(X, L, d, Wg, Wu, N, s2part, run_if_gt, threshold, st);
+    if (rc != POP_OK) return rc;
+    sum_ranges_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2part, pop_prefill_s2_gemm_splits(L), N, s2, run_if_gt, threshold);
     POP_LAUNCHED();
     return POP_OK;
 }
 
 int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
                                double* s2part, double* s2, cudaStream_t st) {
-    if (N <= 0) return POP_OK;
-    static const int kt_env = getenv("POP_PREFILL_KT") ? atoi(getenv("POP_PREFILL_KT")) : 32;
-    int rc;
-    if (dt == POP_F32) rc = launch_s2_gemm<float, G2_KT>(X, L, d, Wg, Wu, N, s2part, st);
-    else if (d % 32 == 0 && kt_env == 32) rc = launch_s2_gemm<__nv_bfloat16, 32>(X, L, d, Wg, Wu, N, s2part, st);
-    else rc = launch_s2_gemm<__nv_bfloat16, G2_KT>(X, L, d, Wg, Wu, N, s2part, st);
-    if (rc != POP_OK) return rc;
-    sum_ranges_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2part, pop_prefill_s2_gemm_splits(L), N, s2);
-    POP_LAUNCHED();
-    return POP_OK;
+    return pop_launch_prefill_s2_gemm_if(X, L, d, Wg, Wu, N, dt, s2part, s2, nullptr, 0, st);
 }
 
 // I_i = sqrt(s2_i) * n_i   (Eq. 3)
@@ -354,14 +363,14 @@ __global__ void __launch_bounds__(PART_NT) partition_kernel(const double* __rest
                                                             int32_t* __restrict__ idx_ret,
                                                             int32_t* __restrict__ idx_cand,
                                                             int32_t* __restrict__ idx_pruned) {
-    __shared__ u32 sm[POP_SELECT_SMEM_WORDS(PART_NT)];
+    __shared__ __align__(8) u32 sm[POP_SELECT_FAST_SMEM_WORDS(PART_NT)];
     const int tid = threadIdx.x;
     const u64* keys = reinterpret_cast<const u64*>(scores);   // non-negative doubles order like their bits
 
     u64 thr1 = ~0ull, thr2 = ~0ull;
     int ne1 = 0, ne2 = 0;
-    if (n_ret > 0) radix_select_kth<PART_NT>(keys, N, n_ret, sm, tid, 0, thr1, ne1);
-    if (n_ret + n_cand > 0) radix_select_kth<PART_NT>(keys, N, n_ret + n_cand, sm, tid, 0, thr2, ne2);
+    if (n_ret > 0) radix_select_kth_fast<PART_NT>(keys, N, n_ret, sm, tid, 0, thr1, ne1);
+    if (n_ret + n_cand > 0) radix_select_kth_fast<PART_NT>(keys, N, n_ret + n_cand, sm, tid, 0, thr2, ne2);
 
     const int per = (N + PART_NT - 1) / PART_NT;
     const int lo = min(N, tid * per), hi = min(N, lo + per);

@@ -1,0 +1,715 @@
+// Prefilling stage on the tensor cores (Sec. 3.3 "Prefilling Stage"; score of Sec. 3.4 Eq. 3), bf16.
+//
+//   H[t, i] = silu(Wg[i].X[t]) * (Wu[i].X[t]),   s2[i] = sum_t H[t, i]^2
+//
+// is a dense contraction over the hidden size (4 L d N flops), so it runs on the 5th-generation
+// tensor cores: tcgen05.mma with the accumulators in tensor memory, operands brought into shared
+// memory by the TMA engine (cp.async.bulk.tensor, 128-byte swizzle) through an mbarrier pipeline.
+//
+// What the partition needs from this pass is a RANKING, and the ranking has to be the one exact
+// arithmetic gives.  So the pass also produces, per channel, a bound of the error of its energy;
+// the few channels whose scores the bounds cannot separate from one of the two rank boundaries
+// (Retained | Candidate, Candidate | Pruned) are then re-scored in fp64 (kernels further down) and
+// the regions are taken on the mixed scores, which rank like exact ones (argument at
+// select_uncertain_kernel).
+//
+// Unit of work: 128 channels (MMA M = tensor-memory lanes) x 128 tokens (MMA N).  With the channels
+// on the lanes one epilogue thread owns one channel and sums over tokens in registers.  The hidden
+// size is consumed in chunks of 128 (8 MMAs of K = 16 each for gate and for up); every chunk starts a
+// fresh accumulator and the epilogue warps add the chunk results in fp32 registers.  That keeps
+// the number of accumulation steps whose rounding is not observable at 8, which is what makes a
+// useful error bound possible (see TC_* constants).  Two accumulator sets (2 x 256 columns) take turns,
+// so the tensor cores work on chunk c + 1 while chunk c is read out.
+//
+// Warp roles (320 threads, one CTA per SM, persistent over units):
+//   warp 0      TMA producer (one lane): Wg tile, Wu tile, X tile of a 64-wide K slab per stage
+//   warp 1      allocates tensor memory; one lane issues the MMAs and the commits
+//   warps 2..9  epilogue: warp w reads lanes 32 (w % 4) .. + 31, columns of token half (w - 2) / 4
+// Every wait is bounded; a wait that runs out sets the status word and the CTA winds down.
+#include <cuda.h>          // CUtensorMap and its enums (the encoder itself is looked up through the runtime)
+
+#include "pop_common.cuh"
+#include "pop_select.cuh"
+
+namespace {
+
+constexpr int TC_BM = 128;                 // channels per unit
+constexpr int TC_BN = 128;                 // tokens per unit
+constexpr int TC_BK = 64;                  // K slab of one pipeline stage: 64 bf16 = one 128-byte swizzle row
+constexpr int TC_STAGES = 4;
+constexpr int TC_CHUNK_SLABS = 2;          // accumulate-restart chunk = 128 hidden dimensions
+constexpr int TC_TILE_BYTES = TC_BM * TC_BK * 2;          // 16 KB
+constexpr int TC_STAGE_BYTES = 3 * TC_TILE_BYTES;         // Wg, Wu, X
+constexpr int TC_THREADS = 320;
+constexpr int TC_EPI_WARPS = 8;
+constexpr int TC_TMEM_COLS = 512;
+constexpr size_t TC_SMEM_BYTES = (size_t)TC_STAGES * TC_STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+
+// Error model of one tcgen05.mma of kind::f16 with an fp32 accumulator (D = C + sum of 16 exact products), as
+// measured on B200 with addends placed around the accumulator's last place: every addend is aligned to the
+// largest one and cut two bits below that one's last place (an addend below 2^-25 of the largest vanishes), the
+// aligned sum is exact, and the result is truncated toward zero to fp32.  Hence
+//   |D - exact| < 16 * 2^-25 * M + 2^-23 * |D|  <=  TC_KAPPA * (sum of the magnitudes of the 17 addends),
+// with M the largest addend and TC_KAPPA = 2^-21 + 2^-23.
+// The sum of magnitudes over one chunk of K is at most |x_chunk|_2 |w_chunk|_2 (Cauchy-Schwarz), and the sum
+// of those over the chunks at most |x|_2 |w|_2.  Adding a chunk result to the running fp32 sum rounds by at
+// most 2^-24 of a sum whose magnitude |x|_2 |w|_2 also bounds.
+constexpr float TC_KAPPA = 5.9604644775390625e-07f;         // 2^-21 + 2^-23
+constexpr float TC_ADD_ULP = 5.9604644775390625e-08f;      // 2^-24
+
+constexpr unsigned long long TC_WAIT_BUDGET_NS = 200ull * 1000ull * 1000ull;   // per wait
+
+enum { TC_ERR_PRODUCER = 101, TC_ERR_MMA_FULL = 102, TC_ERR_MMA_ACC = 103, TC_ERR_EPILOGUE = 104 };
+
+__device__ __forceinline__ u32 smem_u32(const void* p) { return (u32)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(u32 bar, u32 count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(u32 bar, u32 bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(u32 bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ u32 mbar_try_wait(u32 bar, u32 parity) {
+    u32 ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Waits for the phase with the given parity to complete; gives up after TC_WAIT_BUDGET_NS or when another
+// role of the CTA has given up.  Returns false in that case (the caller leaves its loop).
+__device__ __forceinline__ bool mbar_wait(u32 bar, u32 parity, volatile int* abort_flag, u32* status, u32 code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (u32 it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 31u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > TC_WAIT_BUDGET_NS) {
+                *abort_flag = 1;
+                atomicCAS(status, 0u, code);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(u32 dst, const CUtensorMap* map, int x, int y, u32 bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<unsigned long long>(map)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T, both operands K-major bf16, fp32 accumulation.
+__device__ __forceinline__ void umma_bf16(u32 d_tmem, u64 a_desc, u64 b_desc, u32 idesc, u32 accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier gets one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(u32 bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld32(u32 taddr, float (&v)[32]) {
+    u32 r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) in the 128-byte swizzle
+// the TMA engine wrote: groups of 8 rows are 1024 bytes apart (stride byte offset), the leading offset is unused
+// for swizzled K-major tiles (set to 1), descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ u64 smem_desc_sw128(u32 addr) {
+    return (u64)((addr & 0x3ffffu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: fp32 accumulator (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1), both K-major
+// (bits 15, 16 = 0), N / 8 at bit 17, M / 16 at bit 24.
+constexpr u32 TC_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((u32)(TC_BN >> 3) << 17) | ((u32)(TC_BM >> 4) << 24);
+
+struct TcParams {
+    int L, d, N;
+    int n_ct, n_tt, n_pad;        // channel tiles, token tiles, n_ct * 128
+    int nk;                       // K slabs of 64
+    const float* xnorm;           // [n_tt * 128]  |X[t]|_2, rounded up; 0 past L
+    const float* gnorm;           // [n_pad]       |Wg[i]|_2, rounded up; 0 past N
+    const float* unorm;           // [n_pad]
+    double* s2part;               // [2 n_tt][n_pad] partial energies (token half h of token tile tt at 2 tt + h)
+    float* bpart;                 // [2 n_tt][n_pad] bounds of their errors
+    u32* status;
+#ifdef POP_TC_DUMP
+    float* dump_g;                // [n_pad][n_tt * 128] raw gate / up sums (debug builds only)
+    float* dump_u;
+#endif
+};
+
+__global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_constant__ CUtensorMap map_x,
+                                                                   const __grid_constant__ CUtensorMap map_g,
+                                                                   const __grid_constant__ CUtensorMap map_u,
+                                                                   const TcParams P) {
+    extern __shared__ unsigned char tc_smem_raw[];
+    __shared__ u32 tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const u32 raw = smem_u32(tc_smem_raw);
+    const u32 tiles = (raw + 1023u) & ~1023u;                      // stage s at tiles + s * TC_STAGE_BYTES
+    const u32 bars = tiles + TC_STAGES * TC_STAGE_BYTES;           // 8-byte mbarriers
+    const u32 bar_full = bars, bar_empty = bars + 8 * TC_STAGES;
+    const u32 bar_acc_full = bars + 16 * TC_STAGES, bar_acc_empty = bar_acc_full + 16, bar_drain = bar_acc_full + 32;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abortp = &abort_flag;
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_acc_full + 8 * b, 1); mbar_init(bar_acc_empty + 8 * b, TC_EPI_WARPS); }
+        mbar_init(bar_drain, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const u32 tmem_base = tmem_base_slot;
+
+    const int n_units = P.n_ct * P.n_tt;
+    const int n_chunks = (P.nk + TC_CHUNK_SLABS - 1) / TC_CHUNK_SLABS;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            u32 ph = 0;
+            bool ok = true;
+            int issued = 0;
+            for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+                const int ct = unit / P.n_tt, tt = unit - ct * P.n_tt;
+                for (int kb = 0; kb < P.nk; ++kb) {
+                    ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, abortp, P.status, TC_ERR_PRODUCER);
+                    if (!ok) break;
+                    const u32 dst = tiles + (u32)s * TC_STAGE_BYTES, bar = bar_full + 8 * s;
+                    mbar_expect_tx(bar, TC_STAGE_BYTES);
+                    tma_load_2d(dst, &map_g, kb * TC_BK, ct * TC_BM, bar);
+                    tma_load_2d(dst + TC_TILE_BYTES, &map_u, kb * TC_BK, ct * TC_BM, bar);
+                    tma_load_2d(dst + 2 * TC_TILE_BYTES, &map_x, kb * TC_BK, tt * TC_BN, bar);
+                    ++issued;
+                    if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // copies already issued still land in this CTA's shared memory: wait for them (bounded) before leaving.
+                // Stage s is the next to fill; the min(issued, STAGES) stages before it may still be in flight.
+                const int back = issued < TC_STAGES ? issued : TC_STAGES;
+                for (int j = 1; j <= back; ++j) {
+                    int sj = s - j;
+                    u32 pj = ph;
+                    if (sj < 0) { sj += TC_STAGES; pj ^= 1u; }
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_full + 8 * sj, pj) && global_ns() - t0 < TC_WAIT_BUDGET_NS) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            int s = 0, buf = 0;
+            u32 ph = 0, accph[2] = {0u, 0u};
+            bool ok = true;
+            for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+                for (int c = 0; c < n_chunks && ok; ++c) {
+                    ok = mbar_wait(bar_acc_empty + 8 * buf, accph[buf] ^ 1u, abortp, P.status, TC_ERR_MMA_ACC);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const u32 d_g = tmem_base + (u32)buf * 256u, d_u = d_g + 128u;
+                    const int kb_end = min(P.nk, (c + 1) * TC_CHUNK_SLABS);
+                    for (int kb = c * TC_CHUNK_SLABS; kb < kb_end; ++kb) {
+                        ok = mbar_wait(bar_full + 8 * s, ph, abortp, P.status, TC_ERR_MMA_FULL);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const u32 base = tiles + (u32)s * TC_STAGE_BYTES;
+                        const u64 dg = smem_desc_sw128(base), du = smem_desc_sw128(base + TC_TILE_BYTES),
+                                  dx = smem_desc_sw128(base + 2 * TC_TILE_BYTES);
+#pragma unroll
+                        for (int k = 0; k < TC_BK / 16; ++k) {
+                            const u32 acc = (kb > c * TC_CHUNK_SLABS || k > 0) ? 1u : 0u;
+                            // one K = 16 step is 32 bytes along the swizzled row: + 2 in the descriptor's 16-byte units
+                            umma_bf16(d_g, dg + 2ull * k, dx + 2ull * k, TC_IDESC, acc);
+                            umma_bf16(d_u, du + 2ull * k, dx + 2ull * k, TC_IDESC, acc);
+                        }
+                        umma_commit(bar_empty + 8 * s);          // the stage is free once these MMAs have read it
+                        if (++s == TC_STAGES) { s = 0; ph ^= 1u; }
+                    }
+                    if (!ok) break;
+                    umma_commit(bar_acc_full + 8 * buf);         // the chunk's accumulators are complete
+                    accph[buf] ^= 1u;
+                    buf ^= 1;
+                }
+            }
+            // nothing of this CTA may still be executing on the tensor cores when tensor memory is given back
+            umma_commit(bar_drain);
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(bar_drain, 0u) && global_ns() - t0 < TC_WAIT_BUDGET_NS) {}
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int ew = warp - 2;
+        const int quarter = warp & 3;                   // tensor-memory lanes this warp may read: 32 quarter .. + 31
+        const int half = ew >> 2;                       // tokens 64 half .. 64 half + 63 of the unit
+        const u32 lane_base = ((u32)(quarter * 32)) << 16;
+        int buf = 0;
+        u32 accph[2] = {0u, 0u};
+        bool ok = true;
+        // per-MMA steps of a chunk and chunk additions, as a relative bound of |x|_2 |w|_2
+        const float eps = (float)(TC_CHUNK_SLABS * (TC_BK / 16)) * TC_KAPPA + (float)n_chunks * TC_ADD_ULP;
+        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+            const int ct = unit / P.n_tt, tt = unit - ct * P.n_tt;
+            float g[64], u[64];
+#pragma unroll
+            for (int j = 0; j < 64; ++j) { g[j] = 0.f; u[j] = 0.f; }
+            for (int c = 0; c < n_chunks; ++c) {
+                ok = mbar_wait(bar_acc_full + 8 * buf, accph[buf], abortp, P.status, TC_ERR_EPILOGUE);
+                if (!ok) break;
+                tc_fence_after();
+                const u32 t_g = tmem_base + lane_base + (u32)buf * 256u + (u32)half * 64u, t_u = t_g + 128u;
+#pragma unroll
+                for (int p = 0; p < 2; ++p) {
+                    float v[32];
+                    tmem_ld32(t_g + 32u * p, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) g[32 * p + j] += v[j];
+                    tmem_ld32(t_u + 32u * p, v);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) u[32 * p + j] += v[j];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+                accph[buf] ^= 1u;
+                buf ^= 1;
+            }
+            if (!ok) break;
+            // h = silu(g) u in fp32, its square summed in fp64, and a bound of what the fp32 pipeline may have lost
+            const int ch = ct * TC_BM + quarter * 32 + lane;
+#ifdef POP_TC_DUMP
+            if (P.dump_g) {
+                const size_t o = (size_t)ch * (P.n_tt * TC_BN) + tt * TC_BN + half * 64;
+#pragma unroll
+                for (int j = 0; j < 64; ++j) { P.dump_g[o + j] = g[j]; P.dump_u[o + j] = u[j]; }
+            }
+#endif
+            const float cg = eps * P.gnorm[ch], cu = eps * P.unorm[ch];
+            const float* xn = P.xnorm + tt * TC_BN + half * 64;
+            double e2 = 0.0;
+            float eb = 0.f;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) {
+                const float at = __ldg(xn + j);
+                const float dg = at * cg, du = at * cu;                 // |g - exact|, |u - exact| at most these
+                const float gj = g[j], uj = u[j];
+                const float e = __expf(-fmaxf(gj, -80.f));
+                const float s = gj * __fdividef(1.f, 1.f + e);          // silu(g)
+                const float h = s * uj;
+                // |silu'| <= 1.1; the fast exponential and division err by a few ulp, growing with |g|;
+                // past g = -80 the clamped exponential differs from the true one by less than |g| 2e-35
+                const float rho = (8.f + 1.2f * fabsf(gj)) * 1.1920929e-07f;
+                const float dh = 1.1f * dg * fabsf(uj) + (fabsf(s) + 1.1f * dg) * du + rho * fabsf(h) + 2e-35f * fabsf(gj * uj);
+                eb += 2.f * fabsf(h) * dh + dh * dh;
+                e2 = fma((double)h, (double)h, e2);
+            }
+            const size_t slot = (size_t)(2 * tt + half) * P.n_pad + ch;
+            P.s2part[slot] = e2;
+            P.bpart[slot] = eb * 1.0001f;                               // covers the fp32 rounding of this sum itself
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Row norms |row|_2 of a [rows, d] bf16 matrix, rounded up (they are used as bounds), zero for the
+// padding rows up to rows_pad.  One warp per row.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) rownorm_up_kernel(const __nv_bfloat16* __restrict__ M, int rows, int rows_pad, int d,
+                                                         float* __restrict__ out) {
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (r >= rows_pad) return;
+    float acc = 0.f;
+    if (r < rows) {
+        const uint4* row = reinterpret_cast<const uint4*>(M + (size_t)r * d);
+        const int nv = d >> 3;
+        for (int v = lane; v < nv; v += 32) {
+            float f[8];
+            Elem<__nv_bfloat16>::unpack(__ldg(row + v), f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc = fmaf(f[j], f[j], acc);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    // fp32 sum of non-negative terms, at most 1024 + 5 additions per chain (rows are at most 32768 elements):
+    // relative error of the sum below 7e-5, of its root below 4e-5
+    if (lane == 0) out[r] = sqrtf(acc) * 1.001f;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sums the partial energies in a fixed order and forms, per channel, the score a_i = sqrt(s2_i) n_i (Eq. 3)
+// with a bound m_i of |a_i - exact score|: |s2 - exact| <= E gives |sqrt(s2) - sqrt(exact)| <= min(sqrt(E), E / sqrt(s2)).
+// The largest bound goes to *m_max (bit pattern of a non-negative double).
+// ---------------------------------------------------------------------------------------------
+__global__ void tc_finish_kernel(const double* __restrict__ s2part, const float* __restrict__ bpart, int n_parts, int n_pad,
+                                 const double* __restrict__ norm, int N, double* __restrict__ scores,
+                                 double* __restrict__ bounds, u64* __restrict__ m_max) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    double m = 0.0;
+    if (i < N) {
+        double s2 = 0.0, E = 0.0;
+        for (int p = 0; p < n_parts; ++p) {
+            s2 += s2part[(size_t)p * n_pad + i];
+            E += (double)bpart[(size_t)p * n_pad + i];
+        }
+        const double r = sqrt(s2);
+        double dr = sqrt(E);
+        if (r > 0.0) dr = fmin(dr, E / r);
+        m = norm[i] * dr * (1.0 + 1e-9);
+        scores[i] = r * norm[i];
+        bounds[i] = m;
+    }
+    // block maximum, then one atomic
+    __shared__ double red[32];
+    for (int off = 16; off; off >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        m = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.0;
+        for (int off = 16; off; off >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, off));
+        if (threadIdx.x == 0) atomicMax(m_max, (u64)__double_as_longlong(m));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Channels that the bounds cannot place.  Let a_i be the streamed scores, m the largest bound, and tau the
+// n-th largest a_i (n = n_ret for the Retained | Candidate boundary, n_ret + n_cand for Candidate | Pruned).
+//   a_i > tau + 2m  =>  exact score > tau + m; every channel whose exact score is at least that has a_j > tau,
+//                       and fewer than n channels do: i is inside the exact top n.
+//   a_i < tau - 2m  =>  exact score < tau - m, while the n channels with a_j >= tau all have exact scores
+//                       >= tau - m: i is outside the exact top n.
+// The channels in between, for either boundary, are listed (ascending) for exact re-scoring.  Ranking all
+// channels by (exact score where re-scored, streamed score elsewhere) then gives the regions of exact
+// arithmetic: a channel outside the window keeps its side whichever scores the others carry, by the same two
+// counts, and inside the window the order is the exact one.
+// When every bound is zero the streamed scores are exact and nothing is listed.
+// ---------------------------------------------------------------------------------------------
+constexpr int SEL_NT = 1024;
+
+__global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* __restrict__ scores, int N, int n_ret, int n_cand,
+                                                                  const u64* __restrict__ m_max, int32_t* __restrict__ list,
+                                                                  int* __restrict__ n_list) {
+    __shared__ __align__(8) u32 sm[POP_SELECT_FAST_SMEM_WORDS(SEL_NT)];
+    const int tid = threadIdx.x;
+    const double m = __longlong_as_double((long long)*m_max);
+    if (!(m > 0.0)) { if (tid == 0) *n_list = 0; return; }
+    const u64* keys = reinterpret_cast<const u64*>(scores);
+    const int n1 = n_ret, n2 = n_ret + n_cand;
+    const bool b1 = n1 > 0 && n1 < N, b2 = n2 > 0 && n2 < N && n2 != n1;
+    u64 t1 = 0, t2 = 0;
+    int ne;
+    if (b1) radix_select_kth_fast<SEL_NT>(keys, N, n1, sm, tid, 0, t1, ne);
+    if (b2) radix_select_kth_fast<SEL_NT>(keys, N, n2, sm, tid, 0, t2, ne);
+    const double tau1 = __longlong_as_double((long long)t1), tau2 = __longlong_as_double((long long)t2);
+    const double w = 2.0 * m * (1.0 + 1e-9);
+    const int per = (N + SEL_NT - 1) / SEL_NT;
+    const int lo = min(N, tid * per), hi = min(N, lo + per);
+    int cnt = 0;
+    for (int i = lo; i < hi; ++i) {
+        const double a = scores[i];
+        cnt += (b1 && fabs(a - tau1) <= w) || (b2 && fabs(a - tau2) <= w);
+    }
+    int tot;
+    int pos = group_excl_scan<SEL_NT>(cnt, sm, tid, 0, tot);
+    for (int i = lo; i < hi; ++i) {
+        const double a = scores[i];
+        if ((b1 && fabs(a - tau1) <= w) || (b2 && fabs(a - tau2) <= w)) list[pos++] = i;
+    }
+    if (tid == 0) *n_list = tot;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exact (fp64) energies of the listed channels.  Work item = 8 listed channels x 32 tokens; the list is short
+// (tens to a few hundred channels), so the items are small to spread them over the SMs.  64 threads; thread
+// (tg, cg) = (tid / 4, tid % 4) computes tokens 2 tg, 2 tg + 1 x channels 2 cg, 2 cg + 1 (gate and up) from
+// doubles staged in shared memory.  The token sum of an item is taken in a fixed order and written to
+// part[listed channel][token block]; rescore_finish_kernel adds the blocks in order.
+// Does nothing when the list is empty or longer than max_list (then the full fp64 pass runs instead).
+// ---------------------------------------------------------------------------------------------
+constexpr int RS_TOK = 32, RS_CH = 8, RS_KT = 32, RS_NT = 64;
+
+__global__ void __launch_bounds__(RS_NT) rescore_list_kernel(const __nv_bfloat16* __restrict__ X, int L, int d,
+                                                             const __nv_bfloat16* __restrict__ Wg,
+                                                             const __nv_bfloat16* __restrict__ Wu,
+                                                             const int32_t* __restrict__ list, const int* __restrict__ n_list,
+                                                             int max_list, int n_tb, double* __restrict__ part) {
+    // double-buffered operand tiles: the next K step's global loads are in flight during the arithmetic
+    __shared__ __align__(16) double Xs[2][RS_KT][RS_TOK];
+    __shared__ __align__(16) double Gs[2][RS_KT][RS_CH];
+    __shared__ __align__(16) double Us[2][RS_KT][RS_CH];
+    __shared__ double Es[RS_TOK][RS_CH + 1];
+    const int n = *n_list;
+    if (n <= 0 || n > max_list) return;
+    const int tid = threadIdx.x, tg = tid >> 2, cg = tid & 3;
+    const int n_grp = (n + RS_CH - 1) / RS_CH;
+    const int items = n_grp * n_tb;
+    const int nk = (d + RS_KT - 1) / RS_KT;
+    // staging roles: two X vectors (token rows xr, xr + 16; 8 hidden dims at xk) and one W vector per thread
+    const int xr = tid >> 2, xk = (tid & 3) * 8;
+    const int wm = tid >> 5, wr = (tid >> 2) & 7, wk = (tid & 3) * 8;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int grp = item / n_tb, tb = item - grp * n_tb;
+        const int t0 = tb * RS_TOK;
+        const __nv_bfloat16* x0 = (t0 + xr < L) ? X + (size_t)(t0 + xr) * d : nullptr;
+        const __nv_bfloat16* x1 = (t0 + xr + 16 < L) ? X + (size_t)(t0 + xr + 16) * d : nullptr;
+        const int li = grp * RS_CH + wr;
+        const __nv_bfloat16* wrow = li < n ? (wm ? Wu : Wg) + (size_t)list[li] * d : nullptr;
+        uint4 rx0, rx1, rw;
+        auto fetch = [&](int ks) {
+            const int k = ks * RS_KT;
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            rx0 = (x0 && k + xk < d) ? __ldg(reinterpret_cast<const uint4*>(x0 + k + xk)) : z;
+            rx1 = (x1 && k + xk < d) ? __ldg(reinterpret_cast<const uint4*>(x1 + k + xk)) : z;
+            rw = (wrow && k + wk < d) ? __ldg(reinterpret_cast<const uint4*>(wrow + k + wk)) : z;
+        };
+        auto stash = [&](int buf) {
+            float f[8];
+            Elem<__nv_bfloat16>::unpack(rx0, f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) Xs[buf][xk + j][xr] = (double)f[j];
+            Elem<__nv_bfloat16>::unpack(rx1, f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) Xs[buf][xk + j][xr + 16] = (double)f[j];
+            Elem<__nv_bfloat16>::unpack(rw, f);
+            double (*dst)[RS_CH] = wm ? Us[buf] : Gs[buf];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) dst[wk + j][wr] = (double)f[j];
+        };
+        double g[2][2] = {{0, 0}, {0, 0}}, u[2][2] = {{0, 0}, {0, 0}};
+        __syncthreads();                       // the previous item's readers of both buffers and of Es are done
+        fetch(0);
+        stash(0);
+        __syncthreads();
+        for (int ks = 0; ks < nk; ++ks) {
+            const int buf = ks & 1;
+            if (ks + 1 < nk) fetch(ks + 1);
+#pragma unroll 8
+            for (int k = 0; k < RS_KT; ++k) {
+                const double2 xv = *reinterpret_cast<const double2*>(&Xs[buf][k][2 * tg]);
+                const double2 gv = *reinterpret_cast<const double2*>(&Gs[buf][k][2 * cg]);
+                const double2 uv = *reinterpret_cast<const double2*>(&Us[buf][k][2 * cg]);
+                g[0][0] = fma(gv.x, xv.x, g[0][0]); g[0][1] = fma(gv.y, xv.x, g[0][1]);
+                g[1][0] = fma(gv.x, xv.y, g[1][0]); g[1][1] = fma(gv.y, xv.y, g[1][1]);
+                u[0][0] = fma(uv.x, xv.x, u[0][0]); u[0][1] = fma(uv.y, xv.x, u[0][1]);
+                u[1][0] = fma(uv.x, xv.y, u[1][0]); u[1][1] = fma(uv.y, xv.y, u[1][1]);
+            }
+            if (ks + 1 < nk) stash(buf ^ 1);   // nobody reads that buffer before the barrier below
+            __syncthreads();
+        }
+        // tokens past L contribute silu(0) * 0 = 0
+#pragma unroll
+        for (int a = 0; a < 2; ++a)
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const double h = silu_f64(g[a][b]) * u[a][b];
+                Es[2 * tg + a][2 * cg + b] = h * h;
+            }
+        __syncthreads();
+        if (tid < RS_CH) {
+            const int lj = grp * RS_CH + tid;
+            if (lj < n) {
+                double s = 0.0;
+#pragma unroll 1
+                for (int r = 0; r < RS_TOK; ++r) s += Es[r][tid];
+                part[(size_t)lj * n_tb + tb] = s;
+            }
+        }
+    }
+}
+
+// Scores of the re-scored channels: exact energy = sum of the token blocks in order, I_i = sqrt(s2_i) n_i, bound 0.
+// With a list longer than max_list every channel was re-scored by the full fp64 pass into s2_full.
+__global__ void rescore_finish_kernel(const int32_t* __restrict__ list, const int* __restrict__ n_list, int max_list,
+                                      const double* __restrict__ part, int n_tb, const double* __restrict__ s2_full,
+                                      const double* __restrict__ norm, int N, double* __restrict__ scores,
+                                      double* __restrict__ bounds) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int n = *n_list;
+    if (n > max_list) {
+        if (i < N) { scores[i] = sqrt(s2_full[i]) * norm[i]; bounds[i] = 0.0; }
+        return;
+    }
+    if (i >= n) return;
+    const int ch = list[i];
+    double s = 0.0;
+    for (int tb = 0; tb < n_tb; ++tb) s += part[(size_t)i * n_tb + tb];
+    scores[ch] = sqrt(s) * norm[ch];
+    bounds[ch] = 0.0;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        (void)cudaGetLastError();
+        return (EncodeTiledFn)f;
+    }();
+    return fn;
+}
+
+// [rows, d] bf16 row-major; box = 64 columns (128 bytes, the swizzle span) x 128 rows; out-of-range elements read as zero
+int make_map(CUtensorMap* map, const void* base, int rows, int d) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) { pop_set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled is not available from this driver"); return POP_ERR_CUDA; }
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)TC_BM};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        pop_set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled rejected the tensor (base must be 16-byte aligned, row pitch a multiple of 16 bytes)");
+        return POP_ERR_CUDA;
+    }
+    return POP_OK;
+}
+
+}  // namespace
+
+#ifdef POP_TC_DUMP
+// Debug builds: the next tensor-core passes also write their raw gate / up sums ([n_pad][n_tt * 128] floats each).
+static float *g_tc_dump_g = nullptr, *g_tc_dump_u = nullptr;
+extern "C" void pop_debug_tc_dump(float* g, float* u) { g_tc_dump_g = g; g_tc_dump_u = u; }
+#endif
+
+bool pop_prefill_tc_supported(int d, pop_dtype_t dt) { return dt == POP_BF16 && d >= TC_BK && d % 8 == 0; }
+
+void pop_prefill_tc_plan(int L, int d, int N, PrefillTcPlan* plan) {
+    plan->n_ct = (N + TC_BM - 1) / TC_BM;
+    plan->n_tt = (L + TC_BN - 1) / TC_BN;
+    plan->n_pad = plan->n_ct * TC_BM;
+    plan->l_pad = plan->n_tt * TC_BN;
+    plan->n_parts = 2 * plan->n_tt;
+    plan->n_tb = (L + RS_TOK - 1) / RS_TOK;
+    plan->max_list = POP_PREFILL_MAX_LIST;
+}
+
+int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
+                          const PrefillTcScratch& s, double* scores, double* bounds, u32* status, int sm_count,
+                          cudaStream_t st) {
+    PrefillTcPlan plan;
+    pop_prefill_tc_plan(L, d, N, &plan);
+    CUtensorMap mx, mg, mu;
+    int rc = make_map(&mx, X, L, d);
+    if (rc == POP_OK) rc = make_map(&mg, Wg, N, d);
+    if (rc == POP_OK) rc = make_map(&mu, Wu, N, d);
+    if (rc != POP_OK) return rc;
+
+    rownorm_up_kernel<<<(plan.l_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)X, L, plan.l_pad, d, s.xnorm);
+    POP_LAUNCHED();
+    rownorm_up_kernel<<<(plan.n_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)Wg, N, plan.n_pad, d, s.gnorm);
+    POP_LAUNCHED();
+    rownorm_up_kernel<<<(plan.n_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)Wu, N, plan.n_pad, d, s.unorm);
+    POP_LAUNCHED();
+    POP_CUDA(cudaMemsetAsync(s.m_max, 0, sizeof(u64), st));
+
+    static thread_local int cfg_dev = -1;
+    int dev = 0;
+    POP_CUDA(cudaGetDevice(&dev));
+    if (cfg_dev != dev) {
+        POP_CUDA(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_BYTES));
+        cfg_dev = dev;
+    }
+    TcParams P;
+    P.L = L; P.d = d; P.N = N;
+    P.n_ct = plan.n_ct; P.n_tt = plan.n_tt; P.n_pad = plan.n_pad;
+    P.nk = (d + TC_BK - 1) / TC_BK;
+    P.xnorm = s.xnorm; P.gnorm = s.gnorm; P.unorm = s.unorm;
+    P.s2part = s.s2part; P.bpart = s.bpart; P.status = status;
+#ifdef POP_TC_DUMP
+    P.dump_g = g_tc_dump_g; P.dump_u = g_tc_dump_u;
+#endif
+    const int units = plan.n_ct * plan.n_tt;
+    const int grid = units < sm_count ? units : sm_count;
+    prefill_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, mg, mu, P);
+    POP_LAUNCHED();
+
+    tc_finish_kernel<<<(N + 255) / 256, 256, 0, st>>>(s.s2part, s.bpart, plan.n_parts, plan.n_pad, norm, N, scores, bounds, s.m_max);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
+int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
+                               int n_ret, int n_cand, const PrefillTcScratch& s, double* scores, double* bounds,
+                               int sm_count, cudaStream_t st) {
+    PrefillTcPlan plan;
+    pop_prefill_tc_plan(L, d, N, &plan);
+    select_uncertain_kernel<<<1, SEL_NT, 0, st>>>(scores, N, n_ret, n_cand, s.m_max, s.list, s.n_list);
+    POP_LAUNCHED();
+    rescore_list_kernel<<<sm_count * 8, RS_NT, 0, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg,
+                                                        (const __nv_bfloat16*)Wu, s.list, s.n_list, plan.max_list,
+                                                        plan.n_tb, s.part);
+    POP_LAUNCHED();
+    // the full fp64 pass runs only when the list is longer than max_list (its blocks return at once otherwise)
+    int rc = pop_launch_prefill_s2_gemm_if(X, L, d, Wg, Wu, N, POP_BF16, s.s2part_full, s.s2_full, s.n_list, plan.max_list, st);
+    if (rc != POP_OK) return rc;
+    rescore_finish_kernel<<<(N + 255) / 256, 256, 0, st>>>(s.list, s.n_list, plan.max_list, s.part, plan.n_tb, s.s2_full,
+                                                           norm, N, scores, bounds);
+    POP_LAUNCHED();
+    return POP_OK;
+}

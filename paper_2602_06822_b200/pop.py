@@ -55,6 +55,7 @@ SIGNATURES = {
     "pop_partition_sizes": (C.c_int, [_P] + [C.POINTER(C.c_int)] * 3),
     "pop_partition_indices": (C.c_int, [_P] + [C.POINTER(_P)] * 3),
     "pop_partition_scores": (C.c_int, [_P, C.POINTER(_P)]),
+    "pop_partition_score_bounds": (C.c_int, [_P, C.POINTER(_P)]),
     "pop_partition_streamed_scores": (C.c_int, [_P, C.POINTER(_P)]),
     "pop_partition_shape": (C.c_int, [_P, C.POINTER(C.c_int), C.POINTER(C.c_int), C.POINTER(C.c_int)]),
     "pop_partition_check": (C.c_int, [_P]),
@@ -173,6 +174,12 @@ class Partition:
         """Prefill importance scores I_i as a host float64 array (synchronises)."""
         p = C.c_void_p()
         _check(lib().pop_partition_scores(self.handle, C.byref(p)), "pop_partition_scores")
+        return self._view(p.value, self.N, "<f8").cpu().numpy()
+
+    def score_bounds(self) -> np.ndarray:
+        """Bound of |scores()[i] - exact I_i| per channel as a host float64 array (synchronises)."""
+        p = C.c_void_p()
+        _check(lib().pop_partition_score_bounds(self.handle, C.byref(p)), "pop_partition_score_bounds")
         return self._view(p.value, self.N, "<f8").cpu().numpy()
 
     def streamed_scores(self):
