@@ -184,6 +184,7 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     const size_t o_keys = plan.take(sizeof(u64) * (size_t)n_cand);
     const size_t o_yacc = plan.take(sizeof(float) * (size_t)POP_MAX_BATCH * d);
     const size_t o_sel = plan.take(sizeof(int32_t) * (size_t)n_cand);
+    const size_t o_rank = plan.take(sizeof(int32_t) * (size_t)N);
     const size_t o_sync = plan.take(sizeof(u32) * SYNC_WORDS);
     const size_t o_wnorm = plan.take(sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1));
     const size_t o_rpart = plan.take(sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1));
@@ -205,7 +206,7 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     p->idx_ret = (int32_t*)(base + o_ret); p->idx_cand = (int32_t*)(base + o_cand); p->idx_pruned = (int32_t*)(base + o_pruned);
     p->scores = (double*)(base + o_scores); p->score_bounds = (double*)(base + o_bounds); p->norm_cand = (double*)(base + o_norm);
     p->h = (float*)(base + o_h); p->keys = (u64*)(base + o_keys); p->y_acc = (float*)(base + o_yacc);
-    p->sel_slots = (int32_t*)(base + o_sel); p->sync = (u32*)(base + o_sync);
+    p->sel_slots = (int32_t*)(base + o_sel); p->rank_tmp = (int32_t*)(base + o_rank); p->sync = (u32*)(base + o_sync);
     p->wnorm_cand = (float*)(base + o_wnorm); p->rpart = (double*)(base + o_rpart);
     e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
@@ -273,6 +274,7 @@ extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg
         sc.xnorm = (float*)(tb + t_xn); sc.gnorm = (float*)(tb + t_gn); sc.unorm = (float*)(tb + t_un);
         sc.s2part = (double*)(tb + t_tp); sc.bpart = (float*)(tb + t_bp); sc.m_max = (u64*)(tb + t_mm);
         sc.list = (int32_t*)(tb + t_list); sc.n_list = (int*)(tb + t_nl); sc.part = (double*)(tb + t_part);
+        sc.rank = p->rank_tmp;
         sc.s2part_full = s2part; sc.s2_full = s2;
         rc = pop_launch_prefill_tc(X, L, d, Wg, Wu, N, norm, sc, p->scores, p->score_bounds, p->sync + SYNC_ERROR, p->sm_count, st);
         if (rc == POP_OK)
@@ -282,7 +284,7 @@ extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg
                   : pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
         if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, p->scores, st);
     }
-    if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->idx_ret, p->idx_cand, p->idx_pruned, st);
+    if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->rank_tmp, p->sm_count, p->idx_ret, p->idx_cand, p->idx_pruned, st);
     if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
                                                          : pop_launch_repack(p, Wg, Wu, Wd, norm, st);
     cudaFreeAsync(tb, st);

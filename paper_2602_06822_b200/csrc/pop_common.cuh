@@ -67,6 +67,7 @@ struct pop_partition {
                                   // (streamed fp32 score, bound of its error) as two 32-bit patterns
     float* y_acc;                 // [POP_MAX_BATCH][d] fp32 accumulator, zero between steps
     int32_t* sel_slots;           // [n_cand] selected candidate slots (ascending), this step
+    int32_t* rank_tmp;            // [N] prefill scratch: rank of every channel by score
     u32* sync;                    // [SYNC_WORDS] counters / flags, see pop_decode*.cu
     int sm_count;
     int coop;                     // device supports cooperative launch
@@ -119,7 +120,9 @@ int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, cons
 int pop_launch_prefill_s2_gemm_if(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
                                   double* s2part, double* s2, const int* run_if_gt, int threshold, cudaStream_t st);
 int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st);
-int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand,
+// rank[i] = position of channel i in the order (score descending, channel id ascending); rank is [N] scratch
+int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, cudaStream_t st);
+int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* rank_tmp /*[N] scratch*/, int sm_count,
                          int32_t* idx_ret, int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);
 int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                       const double* norm /*[N]*/, cudaStream_t st);
@@ -138,6 +141,7 @@ struct PrefillTcScratch {
     u64* m_max;            // largest score bound (bits of a double)
     int32_t* list;         // [N] channels to re-score
     int* n_list;
+    int32_t* rank;         // [N] rank of every channel by streamed score
     double* part;          // [max_list][n_tb]
     double* s2part_full;   // [pop_prefill_s2_gemm_splits(L)][N]
     double* s2_full;       // [N]

@@ -351,58 +351,98 @@ int pop_launch_scores(const double* s2, const double* norm, int N, double* score
 }
 
 // ---------------------------------------------------------------------------------------------
-// Partition (Sec. 3.3): rank by (score descending, channel id ascending); the first n_ret
-// channels are Retained, the next n_cand Candidate, the rest Pruned.  One block: two radix
-// selects give the two rank boundaries (the tau_high and tau_low thresholds of the paper, with
-// ties split by channel id), then one ordered walk writes the three ascending index lists.
+// Partition (Sec. 3.3): rank by (score descending, channel id ascending); the first n_ret channels are Retained,
+// the next n_cand Candidate, the rest Pruned: the tau_high and tau_low thresholds of the paper taken by rank, with
+// ties split by channel id.
+//
+// Ranks by counting: rank[i] = #{j : key_j > key_i} + #{j < i : key_j == key_i}, the channel's position in that
+// total order.  N^2 comparisons are little work for the whole GPU (N = 11008: 121 M) and need no atomics on shared
+// histogram bins, which is where a single-block radix select spends its time when the keys are the scores of
+// similar channels.  Block (x, y): 512 channels i (two per thread) against the y-th slice of the j range, staged
+// in shared memory; the partial counts meet in rank[] (zeroed by the caller) through one atomic per channel and block.
 // ---------------------------------------------------------------------------------------------
+#define RANK_NT 256
+#define RANK_TILE 1024
+
+__global__ void __launch_bounds__(RANK_NT) rank_kernel(const u64* __restrict__ keys, int N, int j_chunk, int32_t* __restrict__ rank) {
+    __shared__ u64 kj[RANK_TILE];
+    const int tid = threadIdx.x;
+    const int i_lo = blockIdx.x * (2 * RANK_NT), i0 = i_lo + tid, i1 = i0 + RANK_NT;
+    const u64 k0 = i0 < N ? keys[i0] : ~0ull, k1 = i1 < N ? keys[i1] : ~0ull;
+    int c0 = 0, c1 = 0;
+    const int j_begin = blockIdx.y * j_chunk, j_end = min(N, j_begin + j_chunk);
+    for (int t0 = j_begin; t0 < j_end; t0 += RANK_TILE) {
+        const int tn = min(RANK_TILE, j_end - t0);
+        __syncthreads();
+        for (int j = tid; j < tn; j += RANK_NT) kj[j] = keys[t0 + j];
+        __syncthreads();
+        if (t0 + tn <= i_lo) {                            // every j of the tile precedes every i of the block: ties count
+#pragma unroll 8
+            for (int j = 0; j < tn; ++j) { const u64 k = kj[j]; c0 += (k >= k0); c1 += (k >= k1); }
+        } else if (t0 >= i_lo + 2 * RANK_NT) {            // every j follows every i: ties do not count
+#pragma unroll 8
+            for (int j = 0; j < tn; ++j) { const u64 k = kj[j]; c0 += (k > k0); c1 += (k > k1); }
+        } else {
+#pragma unroll 4
+            for (int j = 0; j < tn; ++j) {
+                const u64 k = kj[j];
+                const int jj = t0 + j;
+                c0 += (k > k0) || (k == k0 && jj < i0);
+                c1 += (k > k1) || (k == k1 && jj < i1);
+            }
+        }
+    }
+    if (i0 < N && c0) atomicAdd(&rank[i0], c0);
+    if (i1 < N && c1) atomicAdd(&rank[i1], c1);
+}
+
+int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, cudaStream_t st) {
+    POP_CUDA(cudaMemsetAsync(rank, 0, sizeof(int32_t) * (size_t)N, st));
+    const int bx = (N + 2 * RANK_NT - 1) / (2 * RANK_NT);
+    int by = (4 * sm_count + bx - 1) / bx;                                   // about four blocks per SM in all
+    const int max_by = (N + RANK_TILE - 1) / RANK_TILE;
+    if (by > max_by) by = max_by;
+    if (by < 1) by = 1;
+    int j_chunk = (N + by - 1) / by;
+    j_chunk = (j_chunk + 255) & ~255;                                        // slice boundaries on multiples of 256
+    by = (N + j_chunk - 1) / j_chunk;
+    rank_kernel<<<dim3(bx, by), RANK_NT, 0, st>>>(reinterpret_cast<const u64*>(scores), N, j_chunk, rank);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
+// The three ascending index lists from the ranks: one block, every thread a contiguous chunk of channel ids.
 #define PART_NT 1024
 
-__global__ void __launch_bounds__(PART_NT) partition_kernel(const double* __restrict__ scores, int N,
-                                                            int n_ret, int n_cand,
+__global__ void __launch_bounds__(PART_NT) partition_kernel(const int32_t* __restrict__ rank, int N, int n_ret, int n_cand,
                                                             int32_t* __restrict__ idx_ret,
                                                             int32_t* __restrict__ idx_cand,
                                                             int32_t* __restrict__ idx_pruned) {
-    __shared__ __align__(8) u32 sm[POP_SELECT_FAST_SMEM_WORDS(PART_NT)];
+    __shared__ u32 sm[POP_SELECT_SMEM_WORDS(PART_NT)];
     const int tid = threadIdx.x;
-    const u64* keys = reinterpret_cast<const u64*>(scores);   // non-negative doubles order like their bits
-
-    u64 thr1 = ~0ull, thr2 = ~0ull;
-    int ne1 = 0, ne2 = 0;
-    if (n_ret > 0) radix_select_kth_fast<PART_NT>(keys, N, n_ret, sm, tid, 0, thr1, ne1);
-    if (n_ret + n_cand > 0) radix_select_kth_fast<PART_NT>(keys, N, n_ret + n_cand, sm, tid, 0, thr2, ne2);
-
     const int per = (N + PART_NT - 1) / PART_NT;
     const int lo = min(N, tid * per), hi = min(N, lo + per);
-    int eq1 = 0, eq2 = 0;
-    for (int i = lo; i < hi; ++i) { u64 k = keys[i]; eq1 += (k == thr1); eq2 += (k == thr2); }
-    int tot;
-    const int eb1 = group_excl_scan<PART_NT>(eq1, sm, tid, 0, tot);
-    const int eb2 = group_excl_scan<PART_NT>(eq2, sm, tid, 0, tot);
-    int cR = 0, cC = 0, cP = 0, e1 = eb1, e2 = eb2;
+    const int n_rc = n_ret + n_cand;
+    int cR = 0, cC = 0, cP = 0;
     for (int i = lo; i < hi; ++i) {
-        u64 k = keys[i];
-        bool top1 = k > thr1, top2 = k > thr2;
-        if (k == thr1) { top1 = e1 < ne1; ++e1; }
-        if (k == thr2) { top2 = e2 < ne2; ++e2; }
-        if (top1) ++cR; else if (top2) ++cC; else ++cP;
+        const int r = rank[i];
+        if (r < n_ret) ++cR; else if (r < n_rc) ++cC; else ++cP;
     }
+    int tot;
     int pR = group_excl_scan<PART_NT>(cR, sm, tid, 0, tot);
     int pC = group_excl_scan<PART_NT>(cC, sm, tid, 0, tot);
     int pP = group_excl_scan<PART_NT>(cP, sm, tid, 0, tot);
-    e1 = eb1; e2 = eb2;
     for (int i = lo; i < hi; ++i) {
-        u64 k = keys[i];
-        bool top1 = k > thr1, top2 = k > thr2;
-        if (k == thr1) { top1 = e1 < ne1; ++e1; }
-        if (k == thr2) { top2 = e2 < ne2; ++e2; }
-        if (top1) idx_ret[pR++] = i; else if (top2) idx_cand[pC++] = i; else idx_pruned[pP++] = i;
+        const int r = rank[i];
+        if (r < n_ret) idx_ret[pR++] = i; else if (r < n_rc) idx_cand[pC++] = i; else idx_pruned[pP++] = i;
     }
 }
 
-int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* idx_ret,
+int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* rank_tmp, int sm_count, int32_t* idx_ret,
                          int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st) {
-    partition_kernel<<<1, PART_NT, 0, st>>>(scores, N, n_ret, n_cand, idx_ret, idx_cand, idx_pruned);
+    const int rc = pop_launch_ranks(scores, N, rank_tmp, sm_count, st);
+    if (rc != POP_OK) return rc;
+    partition_kernel<<<1, PART_NT, 0, st>>>(rank_tmp, N, n_ret, n_cand, idx_ret, idx_cand, idx_pruned);
     POP_LAUNCHED();
     return POP_OK;
 }

@@ -443,133 +443,158 @@ __global__ void tc_finish_kernel(const double* __restrict__ s2part, const float*
 // ---------------------------------------------------------------------------------------------
 constexpr int SEL_NT = 1024;
 
-__global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* __restrict__ scores, int N, int n_ret, int n_cand,
+__global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* __restrict__ scores,
+                                                                  const double* __restrict__ bounds,
+                                                                  const int32_t* __restrict__ rank, int N, int n_ret, int n_cand,
                                                                   const u64* __restrict__ m_max, int32_t* __restrict__ list,
                                                                   int* __restrict__ n_list) {
-    __shared__ __align__(8) u32 sm[POP_SELECT_FAST_SMEM_WORDS(SEL_NT)];
+    __shared__ u32 sm[POP_SELECT_SMEM_WORDS(SEL_NT)];
+    __shared__ u64 mw_bits[2];
+    __shared__ double tau_sm[2];
     const int tid = threadIdx.x;
     const double m = __longlong_as_double((long long)*m_max);
     if (!(m > 0.0)) { if (tid == 0) *n_list = 0; return; }
-    const u64* keys = reinterpret_cast<const u64*>(scores);
     const int n1 = n_ret, n2 = n_ret + n_cand;
     const bool b1 = n1 > 0 && n1 < N, b2 = n2 > 0 && n2 < N && n2 != n1;
-    u64 t1 = 0, t2 = 0;
-    int ne;
-    if (b1) radix_select_kth_fast<SEL_NT>(keys, N, n1, sm, tid, 0, t1, ne);
-    if (b2) radix_select_kth_fast<SEL_NT>(keys, N, n2, sm, tid, 0, t2, ne);
-    const double tau1 = __longlong_as_double((long long)t1), tau2 = __longlong_as_double((long long)t2);
-    const double w = 2.0 * m * (1.0 + 1e-9);
     const int per = (N + SEL_NT - 1) / SEL_NT;
     const int lo = min(N, tid * per), hi = min(N, lo + per);
+    if (tid < 2) { mw_bits[tid] = 0ull; tau_sm[tid] = 0.0; }
+    __syncthreads();
+    // tau = the streamed score of the channel at rank n - 1 (exactly one channel holds each rank)
+    for (int i = lo; i < hi; ++i) {
+        const int r = rank[i];
+        if (b1 && r == n1 - 1) tau_sm[0] = scores[i];
+        if (b2 && r == n2 - 1) tau_sm[1] = scores[i];
+    }
+    __syncthreads();
+    const double tau1 = tau_sm[0], tau2 = tau_sm[1];
+    // Outside tau +- 2m every channel is placed (argument above).  Inside, the test can use the channel's own bound:
+    // with m_W the largest bound inside that window, at most n - 1 channels have a_j + m_j > tau + m_W and at least
+    // n have a_j - m_j >= tau - m_W, so a_i - m_i > tau + m_W places i inside the top n and a_i + m_i < tau - m_W
+    // outside, by the same two counts.
+    const double w = 2.0 * m * (1.0 + 1e-9);
+    double mw1 = 0.0, mw2 = 0.0;
+    for (int i = lo; i < hi; ++i) {
+        const double a = scores[i], mi = bounds[i];
+        if (b1 && fabs(a - tau1) <= w) mw1 = fmax(mw1, mi);
+        if (b2 && fabs(a - tau2) <= w) mw2 = fmax(mw2, mi);
+    }
+    if (mw1 > 0.0) atomicMax(&mw_bits[0], (u64)__double_as_longlong(mw1));
+    if (mw2 > 0.0) atomicMax(&mw_bits[1], (u64)__double_as_longlong(mw2));
+    __syncthreads();
+    mw1 = __longlong_as_double((long long)mw_bits[0]) * (1.0 + 1e-9);
+    mw2 = __longlong_as_double((long long)mw_bits[1]) * (1.0 + 1e-9);
     int cnt = 0;
     for (int i = lo; i < hi; ++i) {
-        const double a = scores[i];
-        cnt += (b1 && fabs(a - tau1) <= w) || (b2 && fabs(a - tau2) <= w);
+        const double a = scores[i], mi = bounds[i];
+        cnt += (b1 && fabs(a - tau1) <= w && fabs(a - tau1) <= mi + mw1) || (b2 && fabs(a - tau2) <= w && fabs(a - tau2) <= mi + mw2);
     }
     int tot;
     int pos = group_excl_scan<SEL_NT>(cnt, sm, tid, 0, tot);
     for (int i = lo; i < hi; ++i) {
-        const double a = scores[i];
-        if ((b1 && fabs(a - tau1) <= w) || (b2 && fabs(a - tau2) <= w)) list[pos++] = i;
+        const double a = scores[i], mi = bounds[i];
+        if ((b1 && fabs(a - tau1) <= w && fabs(a - tau1) <= mi + mw1) || (b2 && fabs(a - tau2) <= w && fabs(a - tau2) <= mi + mw2)) list[pos++] = i;
     }
     if (tid == 0) *n_list = tot;
 }
 
 // ---------------------------------------------------------------------------------------------
-// Exact (fp64) energies of the listed channels.  Work item = 8 listed channels x 32 tokens; the list is short
-// (tens to a few hundred channels), so the items are small to spread them over the SMs.  64 threads; thread
-// (tg, cg) = (tid / 4, tid % 4) computes tokens 2 tg, 2 tg + 1 x channels 2 cg, 2 cg + 1 (gate and up) from
-// doubles staged in shared memory.  The token sum of an item is taken in a fixed order and written to
-// part[listed channel][token block]; rescore_finish_kernel adds the blocks in order.
+// Exact (fp64) energies of the listed channels on the fp64 matrix path (mma.m8n8k4.f64: D[8x8] += A[8x4] B[4x8],
+// every product and sum an IEEE fp64 fused multiply-add).  A warp owns 32 tokens (4 A fragments) x 8 listed
+// channels (one B fragment each for their gate and up rows) over the whole hidden size.  Lane (r, c) =
+// (lane / 4, lane % 4) holds row r, k slot c of each fragment; within a block of 32 hidden dimensions slot c is
+// fed from dimensions 8c .. 8c+7, one per step (a dot product does not care in which order its terms are taken
+// as long as both operands agree), so one 16-byte load per row and lane feeds 8 steps, straight from L2 with no
+// shared memory: 6 conversions per 8 matrix instructions.
+// The token sum of an item is taken in a fixed order and written to part[listed channel][token group];
+// rescore_finish_kernel adds the groups in order.
 // Does nothing when the list is empty or longer than max_list (then the full fp64 pass runs instead).
 // ---------------------------------------------------------------------------------------------
-constexpr int RS_TOK = 32, RS_CH = 8, RS_KT = 32, RS_NT = 64;
+constexpr int RS_CH = 8, RS_TOK = 32, RS_WARPS = 4;
 
-__global__ void __launch_bounds__(RS_NT) rescore_list_kernel(const __nv_bfloat16* __restrict__ X, int L, int d,
-                                                             const __nv_bfloat16* __restrict__ Wg,
-                                                             const __nv_bfloat16* __restrict__ Wu,
-                                                             const int32_t* __restrict__ list, const int* __restrict__ n_list,
-                                                             int max_list, int n_tb, double* __restrict__ part) {
-    // double-buffered operand tiles: the next K step's global loads are in flight during the arithmetic
-    __shared__ __align__(16) double Xs[2][RS_KT][RS_TOK];
-    __shared__ __align__(16) double Gs[2][RS_KT][RS_CH];
-    __shared__ __align__(16) double Us[2][RS_KT][RS_CH];
-    __shared__ double Es[RS_TOK][RS_CH + 1];
+__device__ __forceinline__ void dmma_884(double& c0, double& c1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                 : "+d"(c0), "+d"(c1)
+                 : "d"(a), "d"(b));
+}
+// element s (0..7) of a vector of 8 bf16 values, exactly, as a double
+__device__ __forceinline__ double bf16x8_elem(const uint4& v, int s) {
+    const u32 w = (s >> 1) == 0 ? v.x : (s >> 1) == 1 ? v.y : (s >> 1) == 2 ? v.z : v.w;
+    return (double)__uint_as_float((s & 1) ? (w & 0xffff0000u) : (w << 16));
+}
+
+__global__ void __launch_bounds__(32 * RS_WARPS) rescore_list_kernel(const __nv_bfloat16* __restrict__ X, int L, int d,
+                                                                      const __nv_bfloat16* __restrict__ Wg,
+                                                                      const __nv_bfloat16* __restrict__ Wu,
+                                                                      const int32_t* __restrict__ list,
+                                                                      const int* __restrict__ n_list, int max_list, int n_tg,
+                                                                      double* __restrict__ part) {
     const int n = *n_list;
     if (n <= 0 || n > max_list) return;
-    const int tid = threadIdx.x, tg = tid >> 2, cg = tid & 3;
+    const int lane = threadIdx.x & 31, r = lane >> 2, c = lane & 3;
     const int n_grp = (n + RS_CH - 1) / RS_CH;
-    const int items = n_grp * n_tb;
-    const int nk = (d + RS_KT - 1) / RS_KT;
-    // staging roles: two X vectors (token rows xr, xr + 16; 8 hidden dims at xk) and one W vector per thread
-    const int xr = tid >> 2, xk = (tid & 3) * 8;
-    const int wm = tid >> 5, wr = (tid >> 2) & 7, wk = (tid & 3) * 8;
-    for (int item = blockIdx.x; item < items; item += gridDim.x) {
-        const int grp = item / n_tb, tb = item - grp * n_tb;
-        const int t0 = tb * RS_TOK;
-        const __nv_bfloat16* x0 = (t0 + xr < L) ? X + (size_t)(t0 + xr) * d : nullptr;
-        const __nv_bfloat16* x1 = (t0 + xr + 16 < L) ? X + (size_t)(t0 + xr + 16) * d : nullptr;
-        const int li = grp * RS_CH + wr;
-        const __nv_bfloat16* wrow = li < n ? (wm ? Wu : Wg) + (size_t)list[li] * d : nullptr;
-        uint4 rx0, rx1, rw;
-        auto fetch = [&](int ks) {
-            const int k = ks * RS_KT;
-            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-            rx0 = (x0 && k + xk < d) ? __ldg(reinterpret_cast<const uint4*>(x0 + k + xk)) : z;
-            rx1 = (x1 && k + xk < d) ? __ldg(reinterpret_cast<const uint4*>(x1 + k + xk)) : z;
-            rw = (wrow && k + wk < d) ? __ldg(reinterpret_cast<const uint4*>(wrow + k + wk)) : z;
-        };
-        auto stash = [&](int buf) {
-            float f[8];
-            Elem<__nv_bfloat16>::unpack(rx0, f);
+    const int items = n_grp * n_tg;
+    const int nkb = (d + 31) >> 5;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    for (int item = blockIdx.x * RS_WARPS + (threadIdx.x >> 5); item < items; item += gridDim.x * RS_WARPS) {
+        const int grp = item / n_tg, tg = item - grp * n_tg;
+        const __nv_bfloat16* xr[4];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) Xs[buf][xk + j][xr] = (double)f[j];
-            Elem<__nv_bfloat16>::unpack(rx1, f);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) Xs[buf][xk + j][xr + 16] = (double)f[j];
-            Elem<__nv_bfloat16>::unpack(rw, f);
-            double (*dst)[RS_CH] = wm ? Us[buf] : Gs[buf];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) dst[wk + j][wr] = (double)f[j];
-        };
-        double g[2][2] = {{0, 0}, {0, 0}}, u[2][2] = {{0, 0}, {0, 0}};
-        __syncthreads();                       // the previous item's readers of both buffers and of Es are done
-        fetch(0);
-        stash(0);
-        __syncthreads();
-        for (int ks = 0; ks < nk; ++ks) {
-            const int buf = ks & 1;
-            if (ks + 1 < nk) fetch(ks + 1);
-#pragma unroll 8
-            for (int k = 0; k < RS_KT; ++k) {
-                const double2 xv = *reinterpret_cast<const double2*>(&Xs[buf][k][2 * tg]);
-                const double2 gv = *reinterpret_cast<const double2*>(&Gs[buf][k][2 * cg]);
-                const double2 uv = *reinterpret_cast<const double2*>(&Us[buf][k][2 * cg]);
-                g[0][0] = fma(gv.x, xv.x, g[0][0]); g[0][1] = fma(gv.y, xv.x, g[0][1]);
-                g[1][0] = fma(gv.x, xv.y, g[1][0]); g[1][1] = fma(gv.y, xv.y, g[1][1]);
-                u[0][0] = fma(uv.x, xv.x, u[0][0]); u[0][1] = fma(uv.y, xv.x, u[0][1]);
-                u[1][0] = fma(uv.x, xv.y, u[1][0]); u[1][1] = fma(uv.y, xv.y, u[1][1]);
-            }
-            if (ks + 1 < nk) stash(buf ^ 1);   // nobody reads that buffer before the barrier below
-            __syncthreads();
+        for (int a = 0; a < 4; ++a) {
+            const int t = tg * RS_TOK + a * 8 + r;
+            xr[a] = t < L ? X + (size_t)t * d + 8 * c : nullptr;
         }
-        // tokens past L contribute silu(0) * 0 = 0
+        const int li = grp * RS_CH + r;
+        const int ch = li < n ? list[li] : -1;
+        const __nv_bfloat16* wg = ch >= 0 ? Wg + (size_t)ch * d + 8 * c : nullptr;
+        const __nv_bfloat16* wu = ch >= 0 ? Wu + (size_t)ch * d + 8 * c : nullptr;
+        double g[4][2], u[4][2];
 #pragma unroll
-        for (int a = 0; a < 2; ++a)
+        for (int a = 0; a < 4; ++a) { g[a][0] = g[a][1] = u[a][0] = u[a][1] = 0.0; }
+        uint4 vx[4], vg, vu;
+        auto fetch = [&](int kb) {
+            const bool in = (kb << 5) + 8 * c < d;          // d is a multiple of 8: a vector is inside or outside
 #pragma unroll
-            for (int b = 0; b < 2; ++b) {
-                const double h = silu_f64(g[a][b]) * u[a][b];
-                Es[2 * tg + a][2 * cg + b] = h * h;
+            for (int a = 0; a < 4; ++a) vx[a] = (xr[a] && in) ? __ldg(reinterpret_cast<const uint4*>(xr[a] + (kb << 5))) : zero;
+            vg = (wg && in) ? __ldg(reinterpret_cast<const uint4*>(wg + (kb << 5))) : zero;
+            vu = (wu && in) ? __ldg(reinterpret_cast<const uint4*>(wu + (kb << 5))) : zero;
+        };
+        fetch(0);
+        for (int kb = 0; kb < nkb; ++kb) {
+            uint4 cx[4];
+#pragma unroll
+            for (int a = 0; a < 4; ++a) cx[a] = vx[a];
+            const uint4 cg = vg, cu = vu;
+            if (kb + 1 < nkb) fetch(kb + 1);                // the next block's loads fly during this block's arithmetic
+#pragma unroll
+            for (int s = 0; s < 8; ++s) {
+                const double gb = bf16x8_elem(cg, s), ub = bf16x8_elem(cu, s);
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    const double xa = bf16x8_elem(cx[a], s);
+                    dmma_884(g[a][0], g[a][1], xa, gb);
+                    dmma_884(u[a][0], u[a][1], xa, ub);
+                }
             }
-        __syncthreads();
-        if (tid < RS_CH) {
-            const int lj = grp * RS_CH + tid;
-            if (lj < n) {
-                double s = 0.0;
-#pragma unroll 1
-                for (int r = 0; r < RS_TOK; ++r) s += Es[r][tid];
-                part[(size_t)lj * n_tb + tb] = s;
-            }
+        }
+        // lane (r, c) holds token row r of each fragment at listed channels 2c, 2c + 1 of the group; tokens past L gave 0.
+        // Token sum: the 4 fragments in the lane, then the 8 token rows (lanes r = 0..7 of the same c) by shuffles.
+        double e0 = 0.0, e1 = 0.0;
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+            const double h0 = silu_f64(g[a][0]) * u[a][0], h1 = silu_f64(g[a][1]) * u[a][1];
+            e0 = fma(h0, h0, e0);
+            e1 = fma(h1, h1, e1);
+        }
+#pragma unroll
+        for (int off = 4; off < 32; off <<= 1) {
+            e0 += __shfl_xor_sync(0xffffffffu, e0, off);
+            e1 += __shfl_xor_sync(0xffffffffu, e1, off);
+        }
+        if (r == 0) {
+            const int l0 = grp * RS_CH + 2 * c;
+            if (l0 < n) part[(size_t)l0 * n_tg + tg] = e0;
+            if (l0 + 1 < n) part[(size_t)(l0 + 1) * n_tg + tg] = e1;
         }
     }
 }
@@ -645,7 +670,7 @@ void pop_prefill_tc_plan(int L, int d, int N, PrefillTcPlan* plan) {
     plan->n_pad = plan->n_ct * TC_BM;
     plan->l_pad = plan->n_tt * TC_BN;
     plan->n_parts = 2 * plan->n_tt;
-    plan->n_tb = (L + RS_TOK - 1) / RS_TOK;
+    plan->n_tb = (L + RS_TOK - 1) / RS_TOK;         // token groups of the list re-scoring kernel
     plan->max_list = POP_PREFILL_MAX_LIST;
 }
 
@@ -699,9 +724,11 @@ int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, cons
                                int sm_count, cudaStream_t st) {
     PrefillTcPlan plan;
     pop_prefill_tc_plan(L, d, N, &plan);
-    select_uncertain_kernel<<<1, SEL_NT, 0, st>>>(scores, N, n_ret, n_cand, s.m_max, s.list, s.n_list);
+    const int rc0 = pop_launch_ranks(scores, N, s.rank, sm_count, st);
+    if (rc0 != POP_OK) return rc0;
+    select_uncertain_kernel<<<1, SEL_NT, 0, st>>>(scores, bounds, s.rank, N, n_ret, n_cand, s.m_max, s.list, s.n_list);
     POP_LAUNCHED();
-    rescore_list_kernel<<<sm_count * 8, RS_NT, 0, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg,
+    rescore_list_kernel<<<sm_count * 4, 32 * RS_WARPS, 0, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg,
                                                         (const __nv_bfloat16*)Wu, s.list, s.n_list, plan.max_list,
                                                         plan.n_tb, s.part);
     POP_LAUNCHED();

@@ -113,101 +113,6 @@ __device__ void radix_select_kth(const u64* keys, int n, int k, u32* sm, int tid
     need_eq = rem;
 }
 
-// The same result for keys that mostly differ (scores of distinct channels): the first digit starts at the highest
-// bit on which the keys differ, so one counting pass usually leaves a bucket of a few keys; as soon as the bucket
-// of the k-th key holds at most NT keys they are gathered into shared memory and ranked directly.
-// sm: POP_SELECT_FAST_SMEM_WORDS(NT) words.
-#define POP_SELECT_FAST_SMEM_WORDS(NT) (256 + 8 + 2 * (NT))
-
-template <int NT>
-__device__ void radix_select_kth_fast(const u64* keys, int n, int k, u32* sm, int tid, int bar,
-                                      u64& thr, int& need_eq) {
-    const int lane = tid & 31;
-    u64 k0 = keys[0], diff = 0;
-    for (int i = tid; i < n; i += NT) diff |= keys[i] ^ k0;
-#pragma unroll
-    for (int off = 16; off; off >>= 1) diff |= __shfl_xor_sync(0xffffffffu, diff, off);
-    group_sync<NT>(bar);
-    if (tid == 0) { sm[256] = 0; sm[257] = 0; }
-    group_sync<NT>(bar);
-    if (lane == 0) {
-        atomicOr(&sm[256], (u32)(diff & 0xffffffffu));
-        atomicOr(&sm[257], (u32)(diff >> 32));
-    }
-    group_sync<NT>(bar);
-    diff = ((u64)sm[257] << 32) | (u64)sm[256];
-    group_sync<NT>(bar);
-    if (!diff) { thr = k0; need_eq = k; return; }          // all keys equal
-    const int top = 63 - __clzll((long long)diff);
-    int shift = top >= 7 ? top - 7 : 0;                     // digit = bits [shift, shift + width)
-    int width = top - shift + 1;
-    u64 mhi = (shift + width >= 64) ? 0ull : (~0ull << (shift + width));   // bits above the digit: equal in all keys
-    u64 prefix = k0 & mhi;
-    int rem = k;
-    u64* gathered = reinterpret_cast<u64*>(sm + 264);       // [NT] (8-byte aligned: sm is a u32 array at an even word)
-    for (;;) {
-        for (int i = tid; i < 256; i += NT) sm[i] = 0;
-        group_sync<NT>(bar);
-        const u32 dmask = (1u << width) - 1u;
-        for (int i = tid; i < n; i += NT) {
-            const u64 key = keys[i];
-            if ((key & mhi) == prefix) atomicAdd(&sm[(u32)(key >> shift) & dmask], 1u);
-        }
-        group_sync<NT>(bar);
-        if (tid < 32) {
-            u32 c[8], tot = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) { c[j] = sm[8 * lane + j]; tot += c[j]; }
-            u32 incl = tot;                                 // inclusive suffix sum over lanes
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                u32 t = __shfl_down_sync(0xffffffffu, incl, off);
-                if (lane + off < 32) incl += t;
-            }
-            const u32 above = incl - tot;
-            if (above < (u32)rem && (u32)rem <= above + tot) {
-                u32 cum = above;
-#pragma unroll
-                for (int j = 7; j >= 0; --j) {
-                    if (cum + c[j] >= (u32)rem) { sm[256] = 8 * lane + j; sm[257] = cum; sm[258] = c[j]; break; }
-                    cum += c[j];
-                }
-            }
-        }
-        group_sync<NT>(bar);
-        const u32 b = sm[256];
-        const int cnt = (int)sm[258];
-        rem -= (int)sm[257];
-        prefix |= (u64)b << shift;
-        mhi |= (u64)dmask << shift;
-        group_sync<NT>(bar);
-        if (shift == 0) { thr = prefix; need_eq = rem; return; }
-        if (cnt <= NT) {
-            // gather the bucket (order is irrelevant for the value of the rem-th largest) and rank it directly
-            if (tid == 0) sm[259] = 0;
-            group_sync<NT>(bar);
-            for (int i = tid; i < n; i += NT) {
-                const u64 key = keys[i];
-                if ((key & mhi) == prefix) gathered[atomicAdd(&sm[259], 1u)] = key;
-            }
-            group_sync<NT>(bar);
-            if (tid < cnt) {
-                const u64 mine = gathered[tid];
-                int gt = 0, eq = 0;
-                for (int j = 0; j < cnt; ++j) { const u64 o = gathered[j]; gt += (o > mine); eq += (o == mine); }
-                if (gt < rem && rem <= gt + eq) { sm[260] = (u32)(mine & 0xffffffffu); sm[261] = (u32)(mine >> 32); sm[262] = (u32)(rem - gt); }
-            }
-            group_sync<NT>(bar);
-            thr = ((u64)sm[261] << 32) | (u64)sm[260];
-            need_eq = (int)sm[262];
-            group_sync<NT>(bar);
-            return;
-        }
-        width = shift >= 8 ? 8 : shift;
-        shift -= width;
-    }
-}
-
 // Membership in the top k given (thr, need_eq) from radix_select_kth: key > thr, or key == thr
 // and fewer than need_eq equal keys precede it.  The walk below gives every thread a
 // contiguous chunk of indices so that "precede" is a prefix count.
