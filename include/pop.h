@@ -48,6 +48,9 @@ typedef struct { double retained, candidate, pruned; } pop_ratios_t;
 /* Opaque, library-owned: repacked weights, region indices, prefill scores, decode scratch. */
 typedef struct pop_partition pop_partition_t;
 
+/* Opaque, library-owned: what a prefill needs from one weight set alone (see pop_weights_prepare). */
+typedef struct pop_weights pop_weights_t;
+
 /* ---- library information (host only) ------------------------------------------------------- */
 const char* pop_version(void);
 const char* pop_status_string(int status);
@@ -90,6 +93,26 @@ int pop_prefill_partition(const void* X, int L, int d,
                           const void* Wg, const void* Wu, const void* Wd, int N,
                           pop_dtype_t dtype, pop_ratios_t ratios,
                           void* cuda_stream, pop_partition_t** out);
+
+/*
+ * The input-independent part of the prefilling stage, once per weight set instead of once per prompt
+ * (Eq. 3 factors into an activation norm and the weight norm ||Wd[:, i]||_2, which does not depend on
+ * the prompt): the column norms of Wd and, for the tensor-core scoring pass, the row norms of Wg and Wu
+ * (they enter its error bounds) and the TMA descriptors of Wg and Wu.
+ *   Wg, Wu [N, d], Wd [d, N] as for pop_prefill_partition.  The object does NOT copy the weights: the
+ *   caller keeps them alive, at the same addresses and unchanged, until pop_weights_destroy.
+ * Enqueues its kernels on `cuda_stream`; later prefills that use the object must be ordered after them
+ * (same stream, or an event).  Allocates a few N-element device arrays.
+ * pop_prefill_partition_prepared(X, L, w, ...) is pop_prefill_partition(X, L, d, Wg, Wu, Wd, N, dtype, ...)
+ * with those statistics taken from `w`: same results, bit for bit.  The current device must be the one
+ * `w` was prepared on (POP_ERR_INVALID_ARG otherwise).  pop_weights_destroy: the caller has synchronised
+ * the work that used the object.
+ */
+int pop_weights_prepare(const void* Wg, const void* Wu, const void* Wd, int N, int d, pop_dtype_t dtype,
+                        void* cuda_stream, pop_weights_t** out);
+int pop_prefill_partition_prepared(const void* X, int L, const pop_weights_t* w, pop_ratios_t ratios,
+                                   void* cuda_stream, pop_partition_t** out);
+int pop_weights_destroy(pop_weights_t* w);
 
 /*
  * Build a partition from caller-chosen regions instead of prefill scores (the regions of

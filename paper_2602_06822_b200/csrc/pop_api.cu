@@ -52,6 +52,25 @@ extern "C" int pop_region_sizes(int N, pop_ratios_t r, int* n_ret, int* n_cand, 
     return POP_OK;
 }
 
+// Device attributes are looked up once per device (the queries are not free on the prefill path).
+namespace {
+struct DeviceInfo { int valid, sm_count, coop, max_smem_optin; };
+const DeviceInfo& device_info(int device) {
+    static DeviceInfo info[64];
+    static std::mutex m;
+    static DeviceInfo fallback;
+    DeviceInfo* d = (device >= 0 && device < 64) ? &info[device] : &fallback;
+    std::lock_guard<std::mutex> lock(m);
+    if (!d->valid) {
+        cudaDeviceGetAttribute(&d->sm_count, cudaDevAttrMultiProcessorCount, device);
+        cudaDeviceGetAttribute(&d->coop, cudaDevAttrCooperativeLaunch, device);
+        cudaDeviceGetAttribute(&d->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+        d->valid = (d != &fallback);
+    }
+    return *d;
+}
+}  // namespace
+
 static bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
 
 static int check_shape(int d, int N, pop_dtype_t dt) {
@@ -151,9 +170,8 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaGetDevice"); free(p); return POP_ERR_CUDA; }
     p->d = d; p->N = N; p->dtype = dt; p->es = dt == POP_F32 ? 4 : 2;
     p->n_ret = n_ret; p->n_cand = n_cand; p->n_pruned = N - n_ret - n_cand; p->n_rc = n_ret + n_cand;
-    cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
-    cudaDeviceGetAttribute(&p->coop, cudaDevAttrCooperativeLaunch, p->device);
-    cudaDeviceGetAttribute(&p->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
+    const DeviceInfo& di = device_info(p->device);
+    p->sm_count = di.sm_count; p->coop = di.coop; p->max_smem_optin = di.max_smem_optin;
     const size_t row = (size_t)d * p->es;
     // POP_DECODE_IMPL (read at every partition creation) picks the decode kernel family.  Unset or "stream": tiled
     // layout + the dataflow kernel of pop_decode_stream.cu for the bf16 shapes it takes (its one-warp selection holds
@@ -175,19 +193,22 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     const size_t o_ret = plan.take(sizeof(int32_t) * (size_t)n_ret);
     const size_t o_cand = plan.take(sizeof(int32_t) * (size_t)n_cand);
     const size_t o_pruned = plan.take(sizeof(int32_t) * (size_t)p->n_pruned);
+    const size_t o_norm = plan.take(sizeof(double) * (size_t)n_cand);
+    const size_t o_keys = plan.take(sizeof(u64) * (size_t)n_cand);
+    const size_t o_sel = plan.take(sizeof(int32_t) * (size_t)n_cand);
+    const size_t o_wnorm = plan.take(sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1));
+    const size_t o_rpart = plan.take(sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1));
+    // everything that must start at zero sits in one run, cleared by one memset
+    const size_t o_zero = plan.total;
     const size_t o_scores = plan.take(sizeof(double) * (size_t)N);
     const size_t o_bounds = plan.take(sizeof(double) * (size_t)N);
-    const size_t o_norm = plan.take(sizeof(double) * (size_t)n_cand);
+    const size_t o_rank = plan.take(sizeof(int32_t) * (size_t)N);
     // (tiled layout: 8 bytes per element of h, the value with the epoch of the step that wrote it)
     const size_t h_bytes = 2 * sizeof(float) * (size_t)POP_MAX_BATCH * (size_t)(p->h_stride > 0 ? p->h_stride : 1);
     const size_t o_h = plan.take(h_bytes);
-    const size_t o_keys = plan.take(sizeof(u64) * (size_t)n_cand);
     const size_t o_yacc = plan.take(sizeof(float) * (size_t)POP_MAX_BATCH * d);
-    const size_t o_sel = plan.take(sizeof(int32_t) * (size_t)n_cand);
-    const size_t o_rank = plan.take(sizeof(int32_t) * (size_t)N);
     const size_t o_sync = plan.take(sizeof(u32) * SYNC_WORDS);
-    const size_t o_wnorm = plan.take(sizeof(float) * 2 * (size_t)(n_cand > 0 ? n_cand : 1));
-    const size_t o_rpart = plan.take(sizeof(double) * 4 * POP_MAX_BATCH * (size_t)(n_cand > 0 ? n_cand : 1));
+    const size_t zero_bytes = plan.total - o_zero;
     p->slab_bytes = plan.total;
     p->slab = slab_take(p->device, plan.total);
     e = p->slab ? cudaSuccess : cudaMalloc(&p->slab, plan.total);
@@ -208,30 +229,73 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     p->h = (float*)(base + o_h); p->keys = (u64*)(base + o_keys); p->y_acc = (float*)(base + o_yacc);
     p->sel_slots = (int32_t*)(base + o_sel); p->rank_tmp = (int32_t*)(base + o_rank); p->sync = (u32*)(base + o_sync);
     p->wnorm_cand = (float*)(base + o_wnorm); p->rpart = (double*)(base + o_rpart);
-    e = cudaMemsetAsync(p->y_acc, 0, sizeof(float) * (size_t)POP_MAX_BATCH * d, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p->sync, 0, sizeof(u32) * SYNC_WORDS, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p->scores, 0, sizeof(double) * (size_t)N, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p->score_bounds, 0, sizeof(double) * (size_t)N, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(p->h, 0, h_bytes, st);
+    e = cudaMemsetAsync(base + o_zero, 0, zero_bytes, st);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMemsetAsync"); partition_free_now(p, st); return POP_ERR_CUDA; }
     *out = p;
     return POP_OK;
 }
 
-extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg, const void* Wu, const void* Wd,
-                                     int N, pop_dtype_t dtype, pop_ratios_t ratios, void* cuda_stream,
-                                     pop_partition_t** out) {
+// Statistics of a weight set into caller-provided device arrays (norm [N]; gnorm, unorm [n_pad] for bf16 with a
+// tensor-core prefill, else unused).
+static int launch_weight_stats(const void* Wg, const void* Wu, const void* Wd, int N, int d, pop_dtype_t dtype,
+                               double* norm, float* gnorm, float* unorm, int n_pad, cudaStream_t st) {
+    int rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
+    if (rc == POP_OK && pop_prefill_tc_supported(d, dtype)) rc = pop_launch_weight_rownorms(Wg, Wu, N, n_pad, d, gnorm, unorm, st);
+    return rc;
+}
+
+extern "C" int pop_weights_prepare(const void* Wg, const void* Wu, const void* Wd, int N, int d, pop_dtype_t dtype,
+                                   void* cuda_stream, pop_weights_t** out) {
     if (!out) return POP_ERR_INVALID_ARG;
     *out = nullptr;
-    if (!X || !Wg || !Wu || !Wd || L <= 0) return POP_ERR_INVALID_ARG;
+    if (!Wg || !Wu || !Wd) return POP_ERR_INVALID_ARG;
     int rc = check_shape(d, N, dtype);
     if (rc != POP_OK) return rc;
-    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd)) return POP_ERR_INVALID_ARG;
-    int n_ret, n_cand, n_pruned;
-    rc = pop_region_sizes(N, ratios, &n_ret, &n_cand, &n_pruned, nullptr);
-    if (rc != POP_OK) return rc;
+    if (!aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd)) return POP_ERR_INVALID_ARG;
+    pop_weights* w = (pop_weights*)calloc(1, sizeof(pop_weights));
+    if (!w) return POP_ERR_ALLOC;
+    cudaError_t e = cudaGetDevice(&w->device);
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaGetDevice"); free(w); return POP_ERR_CUDA; }
+    w->d = d; w->N = N; w->dtype = dtype; w->Wg = Wg; w->Wu = Wu; w->Wd = Wd;
+    const bool tc = pop_prefill_tc_supported(d, dtype);
+    PrefillTcPlan tp;
+    pop_prefill_tc_plan(1, d, N, &tp);
+    SlabPlan plan;
+    const size_t o_norm = plan.take(sizeof(double) * (size_t)N);
+    const size_t o_gn = plan.take(tc ? sizeof(float) * (size_t)tp.n_pad : 0);
+    const size_t o_un = plan.take(tc ? sizeof(float) * (size_t)tp.n_pad : 0);
+    e = cudaMalloc(&w->block, plan.total);
+    if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMalloc"); free(w); return e == cudaErrorMemoryAllocation ? POP_ERR_ALLOC : POP_ERR_CUDA; }
+    unsigned char* base = (unsigned char*)w->block;
+    w->norm = (double*)(base + o_norm);
+    w->gnorm = tc ? (float*)(base + o_gn) : nullptr;
+    w->unorm = tc ? (float*)(base + o_un) : nullptr;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    rc = launch_weight_stats(Wg, Wu, Wd, N, d, dtype, w->norm, w->gnorm, w->unorm, tp.n_pad, st);
+    if (rc == POP_OK && tc) {
+        rc = pop_prefill_tc_encode_weight_maps(Wg, Wu, N, d, w->map_g, w->map_u);
+        w->have_maps = rc == POP_OK;
+    }
+    if (rc != POP_OK) { cudaStreamSynchronize(st); cudaFree(w->block); free(w); return rc; }
+    *out = w;
+    return POP_OK;
+}
 
+extern "C" int pop_weights_destroy(pop_weights_t* w) {
+    if (!w) return POP_ERR_INVALID_ARG;
+    if (w->block) cudaFree(w->block);
+    free(w);
+    return POP_OK;
+}
+
+// The prefilling stage proper.  `prepared` (may be NULL) carries the statistics of the weight set; without it they
+// are computed into this call's temporaries.
+static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, const void* Wu, const void* Wd, int N,
+                                  pop_dtype_t dtype, pop_ratios_t ratios, const pop_weights* prepared, cudaStream_t st,
+                                  pop_partition_t** out) {
+    int n_ret, n_cand, n_pruned;
+    int rc = pop_region_sizes(N, ratios, &n_ret, &n_cand, &n_pruned, nullptr);
+    if (rc != POP_OK) return rc;
     pop_partition* p = nullptr;
     rc = partition_alloc(d, N, dtype, n_ret, n_cand, st, &p);
     if (rc != POP_OK) return rc;
@@ -243,14 +307,14 @@ extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg
     PrefillTcPlan tp;
     pop_prefill_tc_plan(L, d, N, &tp);
     SlabPlan tmp;
-    const size_t t_norm = tmp.take(sizeof(double) * (size_t)N);
-    const size_t t_s2 = tmp.take(sizeof(double) * (size_t)N);
+    const size_t t_norm = tmp.take(prepared ? 0 : sizeof(double) * (size_t)N);
+    const size_t t_s2 = tmp.take(tc ? 0 : sizeof(double) * (size_t)N);
     const size_t t_s2part = tmp.take(gemm ? sizeof(double) * (size_t)N * (size_t)pop_prefill_s2_gemm_splits(L) : 0);
     size_t t_xn = 0, t_gn = 0, t_un = 0, t_tp = 0, t_bp = 0, t_mm = 0, t_list = 0, t_nl = 0, t_part = 0;
     if (tc) {
         t_xn = tmp.take(sizeof(float) * (size_t)tp.l_pad);
-        t_gn = tmp.take(sizeof(float) * (size_t)tp.n_pad);
-        t_un = tmp.take(sizeof(float) * (size_t)tp.n_pad);
+        t_gn = tmp.take(prepared ? 0 : sizeof(float) * (size_t)tp.n_pad);
+        t_un = tmp.take(prepared ? 0 : sizeof(float) * (size_t)tp.n_pad);
         t_tp = tmp.take(sizeof(double) * (size_t)tp.n_parts * tp.n_pad);
         t_bp = tmp.take(sizeof(float) * (size_t)tp.n_parts * tp.n_pad);
         t_mm = tmp.take(sizeof(u64));
@@ -265,32 +329,65 @@ extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg
         partition_free_now(p, st);
         return POP_ERR_ALLOC;
     }
-    double* norm = (double*)(tb + t_norm);
-    double* s2 = (double*)(tb + t_s2);
+    WeightStats ws;
+    if (prepared) {
+        ws.norm = prepared->norm; ws.gnorm = prepared->gnorm; ws.unorm = prepared->unorm;
+        ws.map_g = prepared->have_maps ? prepared->map_g : nullptr;
+        ws.map_u = prepared->have_maps ? prepared->map_u : nullptr;
+    } else {
+        double* norm = (double*)(tb + t_norm);
+        float *gn = (float*)(tb + t_gn), *un = (float*)(tb + t_un);
+        rc = launch_weight_stats(Wg, Wu, Wd, N, d, dtype, norm, gn, un, tp.n_pad, st);
+        ws.norm = norm; ws.gnorm = gn; ws.unorm = un; ws.map_g = nullptr; ws.map_u = nullptr;
+    }
     double* s2part = (double*)(tb + t_s2part);
-    rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
     if (rc == POP_OK && tc) {
         PrefillTcScratch sc;
-        sc.xnorm = (float*)(tb + t_xn); sc.gnorm = (float*)(tb + t_gn); sc.unorm = (float*)(tb + t_un);
+        sc.xnorm = (float*)(tb + t_xn); sc.gnorm = nullptr; sc.unorm = nullptr;
         sc.s2part = (double*)(tb + t_tp); sc.bpart = (float*)(tb + t_bp); sc.m_max = (u64*)(tb + t_mm);
         sc.list = (int32_t*)(tb + t_list); sc.n_list = (int*)(tb + t_nl); sc.part = (double*)(tb + t_part);
         sc.rank = p->rank_tmp;
-        sc.s2part_full = s2part; sc.s2_full = s2;
-        rc = pop_launch_prefill_tc(X, L, d, Wg, Wu, N, norm, sc, p->scores, p->score_bounds, p->sync + SYNC_ERROR, p->sm_count, st);
+        sc.s2part_full = s2part;
+        rc = pop_launch_prefill_tc(X, L, d, Wg, Wu, N, ws, sc, p->scores, p->score_bounds, p->sync + SYNC_ERROR, p->sm_count, st);
         if (rc == POP_OK)
-            rc = pop_launch_prefill_rescore(X, L, d, Wg, Wu, N, norm, n_ret, n_cand, sc, p->scores, p->score_bounds, p->sm_count, st);
+            rc = pop_launch_prefill_rescore(X, L, d, Wg, Wu, N, ws.norm, n_ret, n_cand, sc, p->scores, p->score_bounds, p->sm_count, st);
     } else if (rc == POP_OK) {
+        double* s2 = (double*)(tb + t_s2);
         rc = gemm ? pop_launch_prefill_s2_gemm(X, L, d, Wg, Wu, N, dtype, s2part, s2, st)
                   : pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
-        if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, p->scores, st);
+        // (rank_tmp is still zero from the partition's creation; scores_kernel clears it all the same)
+        if (rc == POP_OK) rc = pop_launch_scores(s2, ws.norm, N, p->scores, p->rank_tmp, st);
     }
     if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->rank_tmp, p->sm_count, p->idx_ret, p->idx_cand, p->idx_pruned, st);
-    if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
-                                                         : pop_launch_repack(p, Wg, Wu, Wd, norm, st);
+    if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, ws.norm, st)
+                                                         : pop_launch_repack(p, Wg, Wu, Wd, ws.norm, st);
     cudaFreeAsync(tb, st);
     if (rc != POP_OK) { partition_free_now(p, st); return rc; }
     *out = p;
     return POP_OK;
+}
+
+extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg, const void* Wu, const void* Wd,
+                                     int N, pop_dtype_t dtype, pop_ratios_t ratios, void* cuda_stream,
+                                     pop_partition_t** out) {
+    if (!out) return POP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!X || !Wg || !Wu || !Wd || L <= 0) return POP_ERR_INVALID_ARG;
+    int rc = check_shape(d, N, dtype);
+    if (rc != POP_OK) return rc;
+    if (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu) || !aligned16(Wd)) return POP_ERR_INVALID_ARG;
+    return prefill_partition_impl(X, L, d, Wg, Wu, Wd, N, dtype, ratios, nullptr, (cudaStream_t)cuda_stream, out);
+}
+
+extern "C" int pop_prefill_partition_prepared(const void* X, int L, const pop_weights_t* w, pop_ratios_t ratios,
+                                              void* cuda_stream, pop_partition_t** out) {
+    if (!out) return POP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!X || !w || L <= 0 || !aligned16(X)) return POP_ERR_INVALID_ARG;
+    int dev = -1;
+    POP_CUDA(cudaGetDevice(&dev));
+    if (dev != w->device) return POP_ERR_INVALID_ARG;
+    return prefill_partition_impl(X, L, w->d, w->Wg, w->Wu, w->Wd, w->N, w->dtype, ratios, w, (cudaStream_t)cuda_stream, out);
 }
 
 extern "C" int pop_partition_from_indices(const void* Wg, const void* Wu, const void* Wd, int N, int d,

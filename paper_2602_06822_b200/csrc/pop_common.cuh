@@ -74,6 +74,31 @@ struct pop_partition {
     int max_smem_optin;
 };
 
+// Input-independent statistics of one weight set (Wg, Wu, Wd): what a prefill needs from the weights alone.
+// The weights themselves are not copied: the caller keeps them alive and unchanged while the object is in use.
+struct pop_weights {
+    int device;
+    int d, N;
+    pop_dtype_t dtype;
+    const void *Wg, *Wu, *Wd;
+    void* block;                  // the one device allocation behind the arrays below
+    double* norm;                 // [N] ||Wd[:, i]||_2 (the weight factor of Eq. 3)
+    float* gnorm;                 // [n_pad] ||Wg[i]||_2 rounded up, 0 past N (bf16 with a tensor-core prefill, else NULL)
+    float* unorm;                 // [n_pad]
+    int have_maps;                // tensor maps of Wg and Wu below are valid
+    alignas(64) unsigned char map_g[128];
+    alignas(64) unsigned char map_u[128];
+};
+
+// What the prefill kernels take of it (pointers may come from a pop_weights or from a call's own temporaries).
+struct WeightStats {
+    const double* norm;
+    const float* gnorm;
+    const float* unorm;
+    const void* map_g;            // encoded tensor maps of Wg / Wu (128 bytes each), or NULL: encode per call
+    const void* map_u;
+};
+
 // sync[] word assignment (contended counters sit on separate 128-byte lines)
 enum { SYNC_BARRIER = 0, SYNC_TICKET = 1, SYNC_ERROR = 2, SYNC_WORK = 3,
        SYNC_EPOCH = 32, SYNC_CAND_DONE = 96,
@@ -119,10 +144,15 @@ int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, cons
 // the same pass, enqueued always but run only when *run_if_gt > threshold (a device-side decision)
 int pop_launch_prefill_s2_gemm_if(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
                                   double* s2part, double* s2, const int* run_if_gt, int threshold, cudaStream_t st);
-int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st);
-// rank[i] = position of channel i in the order (score descending, channel id ascending); rank is [N] scratch
+// only the blocked pass (no sum over the token ranges), gated the same way
+int pop_launch_prefill_s2_gemm_parts_if(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
+                                        double* s2part, const int* run_if_gt, int threshold, cudaStream_t st);
+// scores[i] = sqrt(s2[i]) * norm[i]; also zeroes rank_to_zero[i] when that is not NULL
+int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, int32_t* rank_to_zero, cudaStream_t st);
+// rank[i] += position of channel i in the order (score descending, channel id ascending); the caller has zeroed rank [N]
+// earlier on the stream (the kernels that write the scores do it: scores_kernel, tc_finish_kernel, rescore_finish_kernel)
 int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, cudaStream_t st);
-int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* rank_tmp /*[N] scratch*/, int sm_count,
+int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* rank_zeroed /*[N]*/, int sm_count,
                          int32_t* idx_ret, int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);
 int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                       const double* norm /*[N]*/, cudaStream_t st);
@@ -144,11 +174,13 @@ struct PrefillTcScratch {
     int32_t* rank;         // [N] rank of every channel by streamed score
     double* part;          // [max_list][n_tb]
     double* s2part_full;   // [pop_prefill_s2_gemm_splits(L)][N]
-    double* s2_full;       // [N]
 };
 bool pop_prefill_tc_supported(int d, pop_dtype_t dt);
 void pop_prefill_tc_plan(int L, int d, int N, PrefillTcPlan* plan);
-int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
+// row norms of Wg and Wu (rounded up, zero past N up to n_pad) in one launch; encoded tensor maps of Wg and Wu
+int pop_launch_weight_rownorms(const void* Wg, const void* Wu, int N, int n_pad, int d, float* gnorm, float* unorm, cudaStream_t st);
+int pop_prefill_tc_encode_weight_maps(const void* Wg, const void* Wu, int N, int d, void* map_g, void* map_u);
+int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const WeightStats& ws,
                           const PrefillTcScratch& s, double* scores, double* bounds, u32* status, int sm_count,
                           cudaStream_t st);
 int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,

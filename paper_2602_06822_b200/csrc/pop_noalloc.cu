@@ -54,6 +54,6 @@ extern "C" int pop_prefill_scores_noalloc(const void* X, int L, int d, const voi
     cudaStream_t st = (cudaStream_t)cuda_stream;
     rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
     if (rc == POP_OK) rc = pop_launch_prefill_s2_exact(X, L, d, Wg, Wu, N, dtype, nullptr, N, s2, st);
-    if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, scores_out, st);
+    if (rc == POP_OK) rc = pop_launch_scores(s2, norm, N, scores_out, nullptr, st);
     return rc;
 }

@@ -318,6 +318,14 @@ static int launch_s2_gemm(const void* X, int L, int d, const void* Wg, const voi
     return POP_OK;
 }
 
+int pop_launch_prefill_s2_gemm_parts_if(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
+                                        double* s2part, const int* run_if_gt, int threshold, cudaStream_t st) {
+    if (N <= 0) return POP_OK;
+    if (dt == POP_F32) return launch_s2_gemm<float, G2_KT>(X, L, d, Wg, Wu, N, s2part, run_if_gt, threshold, st);
+    if (d % 32 == 0) return launch_s2_gemm<__nv_bfloat16, 32>(X, L, d, Wg, Wu, N, s2part, run_if_gt, threshold, st);
+    return launch_s2_gemm<__nv_bfloat16, G2_KT>(X, L, d, Wg, Wu, N, s2part, run_if_gt, threshold, st);
+}
+
 int pop_launch_prefill_s2_gemm_if(const void* X, int L, int d, const void* Wg, const void* Wu, int N, pop_dtype_t dt,
                                   double* s2part, double* s2, const int* run_if_gt, int threshold, cudaStream_t st) {
     if (N <= 0) return POP_OK;
@@ -339,13 +347,16 @@ int pop_launch_prefill_s2_gemm(const void* X, int L, int d, const void* Wg, cons
 
 // I_i = sqrt(s2_i) * n_i   (Eq. 3)
 __global__ void scores_kernel(const double* __restrict__ s2, const double* __restrict__ norm, int N,
-                              double* __restrict__ scores) {
+                              double* __restrict__ scores, int32_t* __restrict__ rank_to_zero) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < N) scores[i] = sqrt(s2[i]) * norm[i];
+    if (i < N) {
+        scores[i] = sqrt(s2[i]) * norm[i];
+        if (rank_to_zero) rank_to_zero[i] = 0;
+    }
 }
 
-int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, cudaStream_t st) {
-    scores_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2, norm, N, scores);
+int pop_launch_scores(const double* s2, const double* norm, int N, double* scores, int32_t* rank_to_zero, cudaStream_t st) {
+    scores_kernel<<<(N + 255) / 256, 256, 0, st>>>(s2, norm, N, scores, rank_to_zero);
     POP_LAUNCHED();
     return POP_OK;
 }
@@ -359,7 +370,7 @@ int pop_launch_scores(const double* s2, const double* norm, int N, double* score
 // total order.  N^2 comparisons are little work for the whole GPU (N = 11008: 121 M) and need no atomics on shared
 // histogram bins, which is where a single-block radix select spends its time when the keys are the scores of
 // similar channels.  Block (x, y): 512 channels i (two per thread) against the y-th slice of the j range, staged
-// in shared memory; the partial counts meet in rank[] (zeroed by the caller) through one atomic per channel and block.
+// in shared memory; the partial counts meet in rank[] (zeroed earlier on the stream) through one atomic per channel and block.
 // ---------------------------------------------------------------------------------------------
 #define RANK_NT 256
 #define RANK_TILE 1024
@@ -397,7 +408,6 @@ __global__ void __launch_bounds__(RANK_NT) rank_kernel(const u64* __restrict__ k
 }
 
 int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, cudaStream_t st) {
-    POP_CUDA(cudaMemsetAsync(rank, 0, sizeof(int32_t) * (size_t)N, st));
     const int bx = (N + 2 * RANK_NT - 1) / (2 * RANK_NT);
     int by = (4 * sm_count + bx - 1) / bx;                                   // about four blocks per SM in all
     const int max_by = (N + RANK_TILE - 1) / RANK_TILE;
@@ -438,7 +448,7 @@ __global__ void __launch_bounds__(PART_NT) partition_kernel(const int32_t* __res
     }
 }
 
-int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* rank_tmp, int sm_count, int32_t* idx_ret,
+int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* rank_tmp /* zeroed */, int sm_count, int32_t* idx_ret,
                          int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st) {
     const int rc = pop_launch_ranks(scores, N, rank_tmp, sm_count, st);
     if (rc != POP_OK) return rc;
@@ -454,20 +464,53 @@ __device__ __forceinline__ int slot_channel(int s, int n_ret, const int32_t* idx
     return s < n_ret ? idx_ret[s] : idx_cand[s - n_ret];
 }
 
-// one block per slot; rows are d*es bytes, a multiple of 16
+// one block per slot; rows are d*es bytes, a multiple of 16.  The block of a candidate slot also leaves the
+// candidate's weight factor of Eq. 3 in norm_cand and, when wmax is given (bf16, streaming decode kernel), the
+// largest magnitudes of its gate and up rows in wmax[0][c], wmax[1][c]: with max |x| they bound any single product
+// of the candidate's dot products (used by the error bound of its streamed score).
 __global__ void __launch_bounds__(256) repack_gu_kernel(const uint4* __restrict__ Wg, const uint4* __restrict__ Wu,
-                                                        int row_vecs, int n_ret,
+                                                        int row_vecs, int n_ret, int n_cand,
                                                         const int32_t* __restrict__ idx_ret,
                                                         const int32_t* __restrict__ idx_cand,
-                                                        uint4* __restrict__ GU) {
+                                                        uint4* __restrict__ GU, const double* __restrict__ norm,
+                                                        double* __restrict__ norm_cand, float* __restrict__ wmax) {
+    __shared__ float red[2][8];
     const int s = blockIdx.x;
     const int ch = slot_channel(s, n_ret, idx_ret, idx_cand);
     const uint4* g = Wg + (size_t)ch * row_vecs;
     const uint4* u = Wu + (size_t)ch * row_vecs;
     uint4* o = GU + (size_t)s * 2 * row_vecs;
+    float mg = 0.f, mu = 0.f;
     for (int v = threadIdx.x; v < row_vecs; v += blockDim.x) {
-        o[v] = g[v];
-        o[row_vecs + v] = u[v];
+        const uint4 a = g[v], b = u[v];
+        o[v] = a;
+        o[row_vecs + v] = b;
+        if (wmax) {                                   // bf16 rows only
+            float f[8];
+            Elem<__nv_bfloat16>::unpack(a, f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mg = fmaxf(mg, fabsf(f[j]));
+            Elem<__nv_bfloat16>::unpack(b, f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mu = fmaxf(mu, fabsf(f[j]));
+        }
+    }
+    if (s < n_ret) return;
+    const int c = s - n_ret;
+    if (threadIdx.x == 0 && norm_cand) norm_cand[c] = norm[ch];
+    if (wmax) {
+#pragma unroll
+        for (int off = 16; off; off >>= 1) {
+            mg = fmaxf(mg, __shfl_xor_sync(0xffffffffu, mg, off));
+            mu = fmaxf(mu, __shfl_xor_sync(0xffffffffu, mu, off));
+        }
+        if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = mg; red[1][threadIdx.x >> 5] = mu; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < 8; ++w) { mg = fmaxf(mg, red[0][w]); mu = fmaxf(mu, red[1][w]); }
+            wmax[c] = mg;
+            wmax[n_cand + c] = mu;
+        }
     }
 }
 
@@ -489,18 +532,12 @@ __global__ void __launch_bounds__(1024) repack_wdt_kernel(const T* __restrict__ 
     if (s < n_rc && j < d) WdT[(size_t)s * d + j] = tile[threadIdx.x][threadIdx.y];
 }
 
-__global__ void gather_norm_kernel(const double* __restrict__ norm, const int32_t* __restrict__ idx_cand,
-                                   int n_cand, double* __restrict__ norm_cand) {
-    int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c < n_cand) norm_cand[c] = norm[idx_cand[c]];
-}
-
 int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                       const double* norm, cudaStream_t st) {
     if (p->n_rc > 0) {
         const int row_vecs = p->d * p->es / 16;
-        repack_gu_kernel<<<p->n_rc, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, p->n_ret,
-                                                  p->idx_ret, p->idx_cand, (uint4*)p->GU);
+        repack_gu_kernel<<<p->n_rc, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, p->n_ret, p->n_cand,
+                                                  p->idx_ret, p->idx_cand, (uint4*)p->GU, norm, p->norm_cand, nullptr);
         POP_LAUNCHED();
         dim3 blk(32, 32), grd((p->n_rc + 31) / 32, (p->d + 31) / 32);
         if (p->dtype == POP_F32)
@@ -512,10 +549,6 @@ int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, co
                                                                    (__nv_bfloat16*)p->WdT);
         POP_LAUNCHED();
     }
-    if (p->n_cand > 0) {
-        gather_norm_kernel<<<(p->n_cand + 255) / 256, 256, 0, st>>>(norm, p->idx_cand, p->n_cand, p->norm_cand);
-        POP_LAUNCHED();
-    }
     return POP_OK;
 }
 
@@ -523,21 +556,23 @@ int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, co
 // Repack into the tiled layout (see pop_common.cuh): the Retained rows as mma.m16n8k16 A
 // fragments, the Candidate rows plain.  One thread writes one 16-byte fragment piece.
 // ---------------------------------------------------------------------------------------------
+// (tiles 0 .. n_rt - 1 hold the retained slots, tiles n_rt .. n_rt + n_ct - 1 the candidate slots)
 __global__ void __launch_bounds__(256) repack_gut_kernel(const __nv_bfloat16* __restrict__ Wg,
-                                                         const __nv_bfloat16* __restrict__ Wu, int d, int n_ret,
-                                                         int n_rt, const int32_t* __restrict__ idx_ret,
-                                                         uint4* __restrict__ GUt) {
+                                                         const __nv_bfloat16* __restrict__ Wu, int d, int n_ret, int n_rt,
+                                                         int n_cand, int n_ct, const int32_t* __restrict__ idx_ret,
+                                                         const int32_t* __restrict__ idx_cand, uint4* __restrict__ GUt) {
     const int KT = d >> 4;
-    const size_t total = (size_t)n_rt * KT * 32;
+    const size_t total = (size_t)(n_rt + n_ct) * KT * 32;
     for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (size_t)gridDim.x * blockDim.x) {
         const int lane = (int)(o & 31);
         const size_t tile = o >> 5;
         const int kt = (int)(tile % KT), rt = (int)(tile / KT);
         const int g = lane >> 2, t = lane & 3;
-        const int slot = 8 * rt + g;
+        const bool cand = rt >= n_rt;
+        const int slot = cand ? 8 * (rt - n_rt) + g : 8 * rt + g;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (slot < n_ret) {
-            const int ch = idx_ret[slot];
+        if (slot < (cand ? n_cand : n_ret)) {
+            const int ch = cand ? idx_cand[slot] : idx_ret[slot];
             const u32* gp = reinterpret_cast<const u32*>(Wg + (size_t)ch * d + (size_t)kt * 16);
             const u32* up = reinterpret_cast<const u32*>(Wu + (size_t)ch * d + (size_t)kt * 16);
             v.x = gp[t];        // row g     (gate), columns 2t, 2t+1
@@ -577,37 +612,21 @@ __global__ void __launch_bounds__(256) repack_wdtt_kernel(const __nv_bfloat16* _
     }
 }
 
-// wmax[0][c] = max |Wg[idx_cand[c]][:]|, wmax[1][c] = max |Wu[idx_cand[c]][:]|: with max |x| they bound any
-// single product of a candidate's dot products (used by the error bound of its streamed score).  One warp per row.
-__global__ void __launch_bounds__(256) rownorm_cand_kernel(const __nv_bfloat16* __restrict__ Wg,
-                                                           const __nv_bfloat16* __restrict__ Wu, int d, int n_cand,
-                                                           const int32_t* __restrict__ idx_cand,
-                                                           float* __restrict__ wmax) {
-    const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (r >= 2 * n_cand) return;
-    const int which = r / n_cand, c = r - which * n_cand;
-    const __nv_bfloat16* row = (which ? Wu : Wg) + (size_t)idx_cand[c] * d;
-    float mx = 0.f;
-    for (int j = lane; j < d; j += 32) mx = fmaxf(mx, fabsf(__bfloat162float(row[j])));
-#pragma unroll
-    for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    if (lane == 0) wmax[r] = mx;
-}
-
 int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                             const double* norm, cudaStream_t st) {
     const size_t row = (size_t)p->d * 2;
     unsigned char* GUt = (unsigned char*)p->GU;
-    unsigned char* GUtc = GUt + (size_t)p->n_rt * 16 * row;            // candidate tiles
     unsigned char* GUc = GUt + (size_t)(p->n_rt + p->n_ct) * 16 * row;  // candidate rows
     unsigned char* WdTt = (unsigned char*)p->WdT;
     unsigned char* WdTc = WdTt + (size_t)p->n_ret_pad * row;
-    if (p->n_rt > 0) {
-        const size_t total = (size_t)p->n_rt * (p->d / 16) * 32;
+    if (p->n_rt + p->n_ct > 0) {
+        const size_t total = (size_t)(p->n_rt + p->n_ct) * (p->d / 16) * 32;
         const int blocks = (int)((total + 255) / 256 < 148 * 64 ? (total + 255) / 256 : 148 * 64);
-        repack_gut_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, p->d, p->n_ret,
-                                                  p->n_rt, p->idx_ret, (uint4*)GUt);
+        repack_gut_kernel<<<blocks, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, p->d, p->n_ret, p->n_rt,
+                                                  p->n_cand, p->n_ct, p->idx_ret, p->idx_cand, (uint4*)GUt);
         POP_LAUNCHED();
+    }
+    if (p->n_rt > 0) {
         const size_t total2 = (size_t)4 * p->n_cg * (p->d / 64) * 32;
         const int blocks2 = (int)((total2 + 255) / 256 < 148 * 64 ? (total2 + 255) / 256 : 148 * 64);
         repack_wdtt_kernel<<<blocks2, 256, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_ret, p->n_cg,
@@ -615,23 +634,13 @@ int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* 
         POP_LAUNCHED();
     }
     if (p->n_cand > 0) {
-        const size_t totalc = (size_t)p->n_ct * (p->d / 16) * 32;
-        const int blocksc = (int)((totalc + 255) / 256 < 148 * 64 ? (totalc + 255) / 256 : 148 * 64);
-        repack_gut_kernel<<<blocksc, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, p->d, p->n_cand,
-                                                   p->n_ct, p->idx_cand, (uint4*)GUtc);
-        POP_LAUNCHED();
-        rownorm_cand_kernel<<<(2 * p->n_cand + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu,
-                                                                      p->d, p->n_cand, p->idx_cand, p->wnorm_cand);
-        POP_LAUNCHED();
         const int row_vecs = (int)(row / 16);
-        repack_gu_kernel<<<p->n_cand, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, 0, p->idx_cand,
-                                                    p->idx_cand, (uint4*)GUc);
+        repack_gu_kernel<<<p->n_cand, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, 0, p->n_cand, p->idx_cand,
+                                                    p->idx_cand, (uint4*)GUc, norm, p->norm_cand, p->wnorm_cand);
         POP_LAUNCHED();
         dim3 blk(32, 32), grd((p->n_cand + 31) / 32, (p->d + 31) / 32);
         repack_wdt_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_cand, 0,
                                                                p->idx_cand, p->idx_cand, (__nv_bfloat16*)WdTc);
-        POP_LAUNCHED();
-        gather_norm_kernel<<<(p->n_cand + 255) / 256, 256, 0, st>>>(norm, p->idx_cand, p->n_cand, p->norm_cand);
         POP_LAUNCHED();
     }
     return POP_OK;

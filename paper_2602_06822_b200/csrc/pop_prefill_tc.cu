@@ -27,6 +27,7 @@
 //   warps 2..9  epilogue: warp w reads lanes 32 (w % 4) .. + 31, columns of token half (w - 2) / 4
 // Every wait is bounded; a wait that runs out sets the status word and the CTA winds down.
 #include <cuda.h>          // CUtensorMap and its enums (the encoder itself is looked up through the runtime)
+#include <string.h>
 
 #include "pop_common.cuh"
 #include "pop_select.cuh"
@@ -368,13 +369,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Row norms |row|_2 of a [rows, d] bf16 matrix, rounded up (they are used as bounds), zero for the
-// padding rows up to rows_pad.  One warp per row.
+// Row norms |row|_2 of [rows, d] bf16 matrices, rounded up (they are used as bounds), zero for the padding rows
+// up to rows_pad.  One warp per row; up to two matrices of the same shape per launch (M1 may be NULL).
+// Thread 0 of the grid also clears the words in zero_a / zero_b when they are given.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) rownorm_up_kernel(const __nv_bfloat16* __restrict__ M, int rows, int rows_pad, int d,
-                                                         float* __restrict__ out) {
-    const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (r >= rows_pad) return;
+__global__ void __launch_bounds__(256) rownorm_up_kernel(const __nv_bfloat16* __restrict__ M0, const __nv_bfloat16* __restrict__ M1,
+                                                         int rows, int rows_pad, int d, float* __restrict__ out0,
+                                                         float* __restrict__ out1, u64* zero_a, int* zero_b) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (zero_a) *zero_a = 0ull;
+        if (zero_b) *zero_b = 0;
+    }
+    int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    const __nv_bfloat16* M = M0;
+    float* out = out0;
+    if (r >= rows_pad) {
+        if (!M1) return;
+        r -= rows_pad; M = M1; out = out1;
+        if (r >= rows_pad) return;
+    }
     float acc = 0.f;
     if (r < rows) {
         const uint4* row = reinterpret_cast<const uint4*>(M + (size_t)r * d);
@@ -400,10 +414,11 @@ __global__ void __launch_bounds__(256) rownorm_up_kernel(const __nv_bfloat16* __
 // ---------------------------------------------------------------------------------------------
 __global__ void tc_finish_kernel(const double* __restrict__ s2part, const float* __restrict__ bpart, int n_parts, int n_pad,
                                  const double* __restrict__ norm, int N, double* __restrict__ scores,
-                                 double* __restrict__ bounds, u64* __restrict__ m_max) {
+                                 double* __restrict__ bounds, u64* __restrict__ m_max, int32_t* __restrict__ rank_to_zero) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     double m = 0.0;
     if (i < N) {
+        rank_to_zero[i] = 0;                      // the ranking pass that follows adds into it
         double s2 = 0.0, E = 0.0;
         for (int p = 0; p < n_parts; ++p) {
             s2 += s2part[(size_t)p * n_pad + i];
@@ -599,16 +614,23 @@ __global__ void __launch_bounds__(32 * RS_WARPS) rescore_list_kernel(const __nv_
     }
 }
 
-// Scores of the re-scored channels: exact energy = sum of the token blocks in order, I_i = sqrt(s2_i) n_i, bound 0.
-// With a list longer than max_list every channel was re-scored by the full fp64 pass into s2_full.
+// Scores of the re-scored channels: exact energy = sum of the token groups in order, I_i = sqrt(s2_i) n_i, bound 0.
+// With a list longer than max_list every channel was re-scored by the full fp64 pass, whose token ranges
+// (s2part_full [n_split][N]) are added here in order.  Also clears rank[] for the ranking pass that follows.
 __global__ void rescore_finish_kernel(const int32_t* __restrict__ list, const int* __restrict__ n_list, int max_list,
-                                      const double* __restrict__ part, int n_tb, const double* __restrict__ s2_full,
-                                      const double* __restrict__ norm, int N, double* __restrict__ scores,
-                                      double* __restrict__ bounds) {
+                                      const double* __restrict__ part, int n_tb, const double* __restrict__ s2part_full,
+                                      int n_split, const double* __restrict__ norm, int N, double* __restrict__ scores,
+                                      double* __restrict__ bounds, int32_t* __restrict__ rank_to_zero) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int n = *n_list;
+    if (i < N) rank_to_zero[i] = 0;
     if (n > max_list) {
-        if (i < N) { scores[i] = sqrt(s2_full[i]) * norm[i]; bounds[i] = 0.0; }
+        if (i < N) {
+            double s = 0.0;
+            for (int y = 0; y < n_split; ++y) s += s2part_full[(size_t)y * N + i];
+            scores[i] = sqrt(s) * norm[i];
+            bounds[i] = 0.0;
+        }
         return;
     }
     if (i >= n) return;
@@ -671,27 +693,44 @@ void pop_prefill_tc_plan(int L, int d, int N, PrefillTcPlan* plan) {
     plan->l_pad = plan->n_tt * TC_BN;
     plan->n_parts = 2 * plan->n_tt;
     plan->n_tb = (L + RS_TOK - 1) / RS_TOK;         // token groups of the list re-scoring kernel
-    plan->max_list = POP_PREFILL_MAX_LIST;
+    // without the blocked fp64 pass (hidden sizes that are not a multiple of 16) the list kernel takes any length
+    plan->max_list = pop_prefill_s2_gemm_supported(d) ? (N < POP_PREFILL_MAX_LIST ? N : POP_PREFILL_MAX_LIST) : N;
 }
 
-int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
+int pop_launch_weight_rownorms(const void* Wg, const void* Wu, int N, int n_pad, int d, float* gnorm, float* unorm, cudaStream_t st) {
+    rownorm_up_kernel<<<(2 * n_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, N, n_pad, d, gnorm,
+                                                           unorm, nullptr, nullptr);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
+int pop_prefill_tc_encode_weight_maps(const void* Wg, const void* Wu, int N, int d, void* map_g, void* map_u) {
+    static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+    int rc = make_map(reinterpret_cast<CUtensorMap*>(map_g), Wg, N, d);
+    if (rc == POP_OK) rc = make_map(reinterpret_cast<CUtensorMap*>(map_u), Wu, N, d);
+    return rc;
+}
+
+int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const WeightStats& ws,
                           const PrefillTcScratch& s, double* scores, double* bounds, u32* status, int sm_count,
                           cudaStream_t st) {
     PrefillTcPlan plan;
     pop_prefill_tc_plan(L, d, N, &plan);
     CUtensorMap mx, mg, mu;
     int rc = make_map(&mx, X, L, d);
-    if (rc == POP_OK) rc = make_map(&mg, Wg, N, d);
-    if (rc == POP_OK) rc = make_map(&mu, Wu, N, d);
     if (rc != POP_OK) return rc;
-
-    rownorm_up_kernel<<<(plan.l_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)X, L, plan.l_pad, d, s.xnorm);
+    if (ws.map_g && ws.map_u) {
+        memcpy(&mg, ws.map_g, sizeof(CUtensorMap));
+        memcpy(&mu, ws.map_u, sizeof(CUtensorMap));
+    } else {
+        rc = make_map(&mg, Wg, N, d);
+        if (rc == POP_OK) rc = make_map(&mu, Wu, N, d);
+        if (rc != POP_OK) return rc;
+    }
+    // token norms; the same launch clears the largest-bound word and the list length
+    rownorm_up_kernel<<<(plan.l_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)X, nullptr, L, plan.l_pad, d, s.xnorm, nullptr,
+                                                            s.m_max, s.n_list);
     POP_LAUNCHED();
-    rownorm_up_kernel<<<(plan.n_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)Wg, N, plan.n_pad, d, s.gnorm);
-    POP_LAUNCHED();
-    rownorm_up_kernel<<<(plan.n_pad + 7) / 8, 256, 0, st>>>((const __nv_bfloat16*)Wu, N, plan.n_pad, d, s.unorm);
-    POP_LAUNCHED();
-    POP_CUDA(cudaMemsetAsync(s.m_max, 0, sizeof(u64), st));
 
     static thread_local int cfg_dev = -1;
     int dev = 0;
@@ -704,7 +743,7 @@ int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const voi
     P.L = L; P.d = d; P.N = N;
     P.n_ct = plan.n_ct; P.n_tt = plan.n_tt; P.n_pad = plan.n_pad;
     P.nk = (d + TC_BK - 1) / TC_BK;
-    P.xnorm = s.xnorm; P.gnorm = s.gnorm; P.unorm = s.unorm;
+    P.xnorm = s.xnorm; P.gnorm = ws.gnorm; P.unorm = ws.unorm;
     P.s2part = s.s2part; P.bpart = s.bpart; P.status = status;
 #ifdef POP_TC_DUMP
     P.dump_g = g_tc_dump_g; P.dump_u = g_tc_dump_u;
@@ -714,7 +753,8 @@ int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const voi
     prefill_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(mx, mg, mu, P);
     POP_LAUNCHED();
 
-    tc_finish_kernel<<<(N + 255) / 256, 256, 0, st>>>(s.s2part, s.bpart, plan.n_parts, plan.n_pad, norm, N, scores, bounds, s.m_max);
+    tc_finish_kernel<<<(N + 255) / 256, 256, 0, st>>>(s.s2part, s.bpart, plan.n_parts, plan.n_pad, ws.norm, N, scores, bounds,
+                                                      s.m_max, s.rank);
     POP_LAUNCHED();
     return POP_OK;
 }
@@ -724,7 +764,7 @@ int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, cons
                                int sm_count, cudaStream_t st) {
     PrefillTcPlan plan;
     pop_prefill_tc_plan(L, d, N, &plan);
-    const int rc0 = pop_launch_ranks(scores, N, s.rank, sm_count, st);
+    const int rc0 = pop_launch_ranks(scores, N, s.rank, sm_count, st);          // s.rank was cleared by tc_finish_kernel
     if (rc0 != POP_OK) return rc0;
     select_uncertain_kernel<<<1, SEL_NT, 0, st>>>(scores, bounds, s.rank, N, n_ret, n_cand, s.m_max, s.list, s.n_list);
     POP_LAUNCHED();
@@ -733,10 +773,12 @@ int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, cons
                                                         plan.n_tb, s.part);
     POP_LAUNCHED();
     // the full fp64 pass runs only when the list is longer than max_list (its blocks return at once otherwise)
-    int rc = pop_launch_prefill_s2_gemm_if(X, L, d, Wg, Wu, N, POP_BF16, s.s2part_full, s.s2_full, s.n_list, plan.max_list, st);
-    if (rc != POP_OK) return rc;
-    rescore_finish_kernel<<<(N + 255) / 256, 256, 0, st>>>(s.list, s.n_list, plan.max_list, s.part, plan.n_tb, s.s2_full,
-                                                           norm, N, scores, bounds);
+    if (plan.max_list < N) {
+        const int rc = pop_launch_prefill_s2_gemm_parts_if(X, L, d, Wg, Wu, N, POP_BF16, s.s2part_full, s.n_list, plan.max_list, st);
+        if (rc != POP_OK) return rc;
+    }
+    rescore_finish_kernel<<<(N + 255) / 256, 256, 0, st>>>(s.list, s.n_list, plan.max_list, s.part, plan.n_tb, s.s2part_full,
+                                                           pop_prefill_s2_gemm_splits(L), norm, N, scores, bounds, s.rank);
     POP_LAUNCHED();
     return POP_OK;
 }

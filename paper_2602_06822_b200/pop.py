@@ -50,6 +50,9 @@ SIGNATURES = {
     "pop_region_sizes": (C.c_int, [C.c_int, Ratios] + [C.POINTER(C.c_int)] * 4),
     "pop_prefill_partition": (C.c_int, [_P, C.c_int, C.c_int, _P, _P, _P, C.c_int, C.c_int, Ratios, _P,
                                         C.POINTER(_P)]),
+    "pop_weights_prepare": (C.c_int, [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P, C.POINTER(_P)]),
+    "pop_prefill_partition_prepared": (C.c_int, [_P, C.c_int, _P, Ratios, _P, C.POINTER(_P)]),
+    "pop_weights_destroy": (C.c_int, [_P]),
     "pop_partition_from_indices": (C.c_int, [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P, C.c_int, _P, C.c_int,
                                              _P, C.POINTER(_P)]),
     "pop_partition_sizes": (C.c_int, [_P] + [C.POINTER(C.c_int)] * 3),
@@ -223,6 +226,51 @@ def prefill_partition(X, Wg, Wu, Wd, ratios, stream=None) -> Partition:
                                        Ratios(*ratios), _stream_ptr(stream), C.byref(out)),
            "pop_prefill_partition")
     return Partition(out.value, X.device)
+
+
+class Weights:
+    """Owner of a ``pop_weights_t*`` (pop_weights_prepare).  Keeps references to the weight tensors, which the
+    library reads again at every prefill that uses the object."""
+
+    def __init__(self, Wg, Wu, Wd, stream=None):
+        for t in (Wg, Wu, Wd):
+            if not (t.is_cuda and t.is_contiguous()):
+                raise ValueError("tensors must be contiguous CUDA tensors")
+        N, d = Wg.shape
+        if tuple(Wu.shape) != (N, d) or tuple(Wd.shape) != (d, N):
+            raise ValueError("shape mismatch")
+        dt = _dtype_code(Wg)
+        if any(_dtype_code(t) != dt for t in (Wu, Wd)):
+            raise TypeError("dtype mismatch")
+        self.tensors = (Wg, Wu, Wd)
+        self.device = Wg.device
+        out = C.c_void_p()
+        _check(lib().pop_weights_prepare(Wg.data_ptr(), Wu.data_ptr(), Wd.data_ptr(), N, d, dt, _stream_ptr(stream),
+                                         C.byref(out)), "pop_weights_prepare")
+        self._h = out
+
+    def prefill_partition(self, X, ratios, stream=None) -> "Partition":
+        """pop_prefill_partition_prepared: X [L, d] -> partition, with this weight set's statistics."""
+        if not (X.is_cuda and X.is_contiguous()) or _dtype_code(X) != _dtype_code(self.tensors[0]):
+            raise ValueError("X must be a contiguous CUDA tensor of the weights' dtype")
+        if X.shape[1] != self.tensors[0].shape[1]:
+            raise ValueError("shape mismatch")
+        out = C.c_void_p()
+        _check(lib().pop_prefill_partition_prepared(X.data_ptr(), X.shape[0], self._h, Ratios(*ratios), _stream_ptr(stream),
+                                                    C.byref(out)), "pop_prefill_partition_prepared")
+        return Partition(out.value, X.device)
+
+    def destroy(self):
+        if self._h is not None:
+            _torch().cuda.synchronize(self.device)
+            lib().pop_weights_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
 
 
 def partition_from_indices(Wg, Wu, Wd, ret: np.ndarray, cand: np.ndarray, stream=None) -> Partition:
