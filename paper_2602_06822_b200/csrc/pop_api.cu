@@ -341,8 +341,8 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
         ws.norm = norm; ws.gnorm = gn; ws.unorm = un; ws.map_g = nullptr; ws.map_u = nullptr;
     }
     double* s2part = (double*)(tb + t_s2part);
+    PrefillTcScratch sc;
     if (rc == POP_OK && tc) {
-        PrefillTcScratch sc;
         sc.xnorm = (float*)(tb + t_xn); sc.gnorm = nullptr; sc.unorm = nullptr;
         sc.s2part = (double*)(tb + t_tp); sc.bpart = (float*)(tb + t_bp); sc.m_max = (u64*)(tb + t_mm);
         sc.list = (int32_t*)(tb + t_list); sc.n_list = (int*)(tb + t_nl); sc.part = (double*)(tb + t_part);
@@ -358,7 +358,10 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
         // (rank_tmp is still zero from the partition's creation; scores_kernel clears it all the same)
         if (rc == POP_OK) rc = pop_launch_scores(s2, ws.norm, N, p->scores, p->rank_tmp, st);
     }
-    if (rc == POP_OK) rc = pop_launch_partition(p->scores, N, n_ret, n_cand, p->rank_tmp, p->sm_count, p->idx_ret, p->idx_cand, p->idx_pruned, st);
+    if (rc == POP_OK)
+        rc = tc ? pop_launch_partition_after_rescore(p->scores, N, n_ret, n_cand, p->rank_tmp, p->sm_count, sc.list, sc.n_list,
+                                                     tp.max_list, p->idx_ret, p->idx_cand, p->idx_pruned, st)
+                : pop_launch_partition(p->scores, N, n_ret, n_cand, p->rank_tmp, p->sm_count, p->idx_ret, p->idx_cand, p->idx_pruned, st);
     if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, ws.norm, st)
                                                          : pop_launch_repack(p, Wg, Wu, Wd, ws.norm, st);
     cudaFreeAsync(tb, st);

@@ -154,6 +154,9 @@ int pop_launch_scores(const double* s2, const double* norm, int N, double* score
 int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, cudaStream_t st);
 int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int32_t* rank_zeroed /*[N]*/, int sm_count,
                          int32_t* idx_ret, int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);
+int pop_launch_partition_after_rescore(const double* scores, int N, int n_ret, int n_cand, int32_t* rank, int sm_count,
+                                       const int32_t* list, const int* n_list, int max_list, int32_t* idx_ret,
+                                       int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st);
 int pop_launch_repack(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                       const double* norm /*[N]*/, cudaStream_t st);
 int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,

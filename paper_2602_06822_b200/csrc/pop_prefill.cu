@@ -375,8 +375,10 @@ int pop_launch_scores(const double* s2, const double* norm, int N, double* score
 #define RANK_NT 256
 #define RANK_TILE 1024
 
-__global__ void __launch_bounds__(RANK_NT) rank_kernel(const u64* __restrict__ keys, int N, int j_chunk, int32_t* __restrict__ rank) {
+__global__ void __launch_bounds__(RANK_NT) rank_kernel(const u64* __restrict__ keys, int N, int j_chunk, int32_t* __restrict__ rank,
+                                                       const int* __restrict__ run_if_gt, int threshold) {
     __shared__ u64 kj[RANK_TILE];
+    if (run_if_gt && *run_if_gt <= threshold) return;           // the same decision in every thread of the grid
     const int tid = threadIdx.x;
     const int i_lo = blockIdx.x * (2 * RANK_NT), i0 = i_lo + tid, i1 = i0 + RANK_NT;
     const u64 k0 = i0 < N ? keys[i0] : ~0ull, k1 = i1 < N ? keys[i1] : ~0ull;
@@ -407,7 +409,34 @@ __global__ void __launch_bounds__(RANK_NT) rank_kernel(const u64* __restrict__ k
     if (i1 < N && c1) atomicAdd(&rank[i1], c1);
 }
 
-int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, cudaStream_t st) {
+// Ranks of the listed channels only (the others keep theirs): rank[list[t]] += number of channels that precede it.
+// Block (x, y): 128 listed channels against the y-th slice of all channels.  Runs when 0 < *n_list <= max_list.
+__global__ void __launch_bounds__(128) rank_list_kernel(const u64* __restrict__ keys, int N, int j_chunk,
+                                                        const int32_t* __restrict__ list, const int* __restrict__ n_list,
+                                                        int max_list, int32_t* __restrict__ rank) {
+    __shared__ u64 kj[RANK_TILE];
+    const int n = *n_list;
+    if (n <= 0 || n > max_list || (int)(blockIdx.x * 128) >= n) return;
+    const int tid = threadIdx.x, t = blockIdx.x * 128 + tid;
+    const int i = t < n ? list[t] : -1;
+    const u64 ki = i >= 0 ? keys[i] : ~0ull;
+    int c = 0;
+    const int j_begin = blockIdx.y * j_chunk, j_end = min(N, j_begin + j_chunk);
+    for (int t0 = j_begin; t0 < j_end; t0 += RANK_TILE) {
+        const int tn = min(RANK_TILE, j_end - t0);
+        __syncthreads();
+        for (int j = tid; j < tn; j += 128) kj[j] = keys[t0 + j];
+        __syncthreads();
+#pragma unroll 4
+        for (int j = 0; j < tn; ++j) {
+            const u64 k = kj[j];
+            c += (k > ki) || (k == ki && t0 + j < i);
+        }
+    }
+    if (i >= 0 && c) atomicAdd(&rank[i], c);
+}
+
+static int launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, const int* run_if_gt, int threshold, cudaStream_t st) {
     const int bx = (N + 2 * RANK_NT - 1) / (2 * RANK_NT);
     int by = (4 * sm_count + bx - 1) / bx;                                   // about four blocks per SM in all
     const int max_by = (N + RANK_TILE - 1) / RANK_TILE;
@@ -416,9 +445,13 @@ int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, c
     int j_chunk = (N + by - 1) / by;
     j_chunk = (j_chunk + 255) & ~255;                                        // slice boundaries on multiples of 256
     by = (N + j_chunk - 1) / j_chunk;
-    rank_kernel<<<dim3(bx, by), RANK_NT, 0, st>>>(reinterpret_cast<const u64*>(scores), N, j_chunk, rank);
+    rank_kernel<<<dim3(bx, by), RANK_NT, 0, st>>>(reinterpret_cast<const u64*>(scores), N, j_chunk, rank, run_if_gt, threshold);
     POP_LAUNCHED();
     return POP_OK;
+}
+
+int pop_launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, cudaStream_t st) {
+    return launch_ranks(scores, N, rank, sm_count, nullptr, 0, st);
 }
 
 // The three ascending index lists from the ranks: one block, every thread a contiguous chunk of channel ids.
@@ -453,6 +486,33 @@ int pop_launch_partition(const double* scores, int N, int n_ret, int n_cand, int
     const int rc = pop_launch_ranks(scores, N, rank_tmp, sm_count, st);
     if (rc != POP_OK) return rc;
     partition_kernel<<<1, PART_NT, 0, st>>>(rank_tmp, N, n_ret, n_cand, idx_ret, idx_cand, idx_pruned);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
+// After a re-scoring of the listed channels: only they can have changed sides of a rank boundary, and a channel that
+// was not listed is on the same side under the mixed scores as under its first rank (argument at
+// select_uncertain_kernel), so only the listed channels are ranked again (their rank entries were cleared by
+// rescore_finish_kernel).  When the list was longer than max_list every score was replaced: then all ranks were
+// cleared and the full ranking runs instead.
+int pop_launch_partition_after_rescore(const double* scores, int N, int n_ret, int n_cand, int32_t* rank, int sm_count,
+                                       const int32_t* list, const int* n_list, int max_list, int32_t* idx_ret,
+                                       int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st) {
+    // lists are short (blocks past the list's end return at once), so the channel axis is cut finely
+    int by = (N + 511) / 512;
+    if (by > 64) by = 64;
+    if (by < 1) by = 1;
+    (void)sm_count;
+    int j_chunk = (((N + by - 1) / by) + 255) & ~255;
+    by = (N + j_chunk - 1) / j_chunk;
+    rank_list_kernel<<<dim3((max_list + 127) / 128, by), 128, 0, st>>>(reinterpret_cast<const u64*>(scores), N, j_chunk, list, n_list,
+                                                                      max_list, rank);
+    POP_LAUNCHED();
+    if (max_list < N) {
+        const int rc = launch_ranks(scores, N, rank, sm_count, n_list, max_list, st);
+        if (rc != POP_OK) return rc;
+    }
+    partition_kernel<<<1, PART_NT, 0, st>>>(rank, N, n_ret, n_cand, idx_ret, idx_cand, idx_pruned);
     POP_LAUNCHED();
     return POP_OK;
 }

@@ -15,9 +15,9 @@
 //
 // Unit of work: 128 channels (MMA M = tensor-memory lanes) x 128 tokens (MMA N).  With the channels
 // on the lanes one epilogue thread owns one channel and sums over tokens in registers.  The hidden
-// size is consumed in chunks of 128 (8 MMAs of K = 16 each for gate and for up); every chunk starts a
+// size is consumed in chunks of 64 (4 MMAs of K = 16 each for gate and for up); every chunk starts a
 // fresh accumulator and the epilogue warps add the chunk results in fp32 registers.  That keeps
-// the number of accumulation steps whose rounding is not observable at 8, which is what makes a
+// the number of accumulation steps whose rounding is not observable at 4, which is what makes a
 // useful error bound possible (see TC_* constants).  Two accumulator sets (2 x 256 columns) take turns,
 // so the tensor cores work on chunk c + 1 while chunk c is read out.
 //
@@ -38,7 +38,8 @@ constexpr int TC_BM = 128;                 // channels per unit
 constexpr int TC_BN = 128;                 // tokens per unit
 constexpr int TC_BK = 64;                  // K slab of one pipeline stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_STAGES = 4;
-constexpr int TC_CHUNK_SLABS = 2;          // accumulate-restart chunk = 128 hidden dimensions
+constexpr int TC_CHUNK_SLABS = 1;          // accumulate-restart chunk = 64 hidden dimensions (4 MMAs)
+constexpr int TC_TRACK = 4;                // the running sums' magnitudes are sampled every TC_TRACK chunks
 constexpr int TC_TILE_BYTES = TC_BM * TC_BK * 2;          // 16 KB
 constexpr int TC_STAGE_BYTES = 3 * TC_TILE_BYTES;         // Wg, Wu, X
 constexpr int TC_THREADS = 320;
@@ -53,8 +54,12 @@ constexpr size_t TC_SMEM_BYTES = (size_t)TC_STAGES * TC_STAGE_BYTES + 1024 /* al
 //   |D - exact| < 16 * 2^-25 * M + 2^-23 * |D|  <=  TC_KAPPA * (sum of the magnitudes of the 17 addends),
 // with M the largest addend and TC_KAPPA = 2^-21 + 2^-23.
 // The sum of magnitudes over one chunk of K is at most |x_chunk|_2 |w_chunk|_2 (Cauchy-Schwarz), and the sum
-// of those over the chunks at most |x|_2 |w|_2.  Adding a chunk result to the running fp32 sum rounds by at
-// most 2^-24 of a sum whose magnitude |x|_2 |w|_2 also bounds.
+// of those over the chunks at most |x|_2 |w|_2: the MMA steps of a dot product err by at most
+// (steps per chunk) * TC_KAPPA * |x|_2 |w|_2 in all.
+// Adding a chunk result to the running fp32 sum rounds by at most 2^-24 of the new sum.  The running sums are
+// observed: every TC_TRACK chunks a thread takes the largest magnitude among its sums; between two samples a sum
+// moves by at most the Cauchy-Schwarz bounds of the chunks in between, so the magnitudes of all n_chunks sums add up
+// to at most TC_TRACK * (sum of the samples + |x|_2 |w|_2).
 constexpr float TC_KAPPA = 5.9604644775390625e-07f;         // 2^-21 + 2^-23
 constexpr float TC_ADD_ULP = 5.9604644775390625e-08f;      // 2^-24
 
@@ -297,13 +302,15 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
         int buf = 0;
         u32 accph[2] = {0u, 0u};
         bool ok = true;
-        // per-MMA steps of a chunk and chunk additions, as a relative bound of |x|_2 |w|_2
-        const float eps = (float)(TC_CHUNK_SLABS * (TC_BK / 16)) * TC_KAPPA + (float)n_chunks * TC_ADD_ULP;
+        // the MMA steps of a chunk, and the part of the chunk additions that the samples do not cover, as a
+        // relative bound of |x|_2 |w|_2
+        const float eps = (float)(TC_CHUNK_SLABS * (TC_BK / 16)) * TC_KAPPA + (float)TC_TRACK * TC_ADD_ULP;
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
             const int ct = unit / P.n_tt, tt = unit - ct * P.n_tt;
             float g[64], u[64];
 #pragma unroll
             for (int j = 0; j < 64; ++j) { g[j] = 0.f; u[j] = 0.f; }
+            float track_g = 0.f, track_u = 0.f;           // sums of the sampled largest |running sum|
             for (int c = 0; c < n_chunks; ++c) {
                 ok = mbar_wait(bar_acc_full + 8 * buf, accph[buf], abortp, P.status, TC_ERR_EPILOGUE);
                 if (!ok) break;
@@ -324,6 +331,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
                 if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
                 accph[buf] ^= 1u;
                 buf ^= 1;
+                if ((c % TC_TRACK) == TC_TRACK - 1 || c == n_chunks - 1) {
+                    float mg = 0.f, mu = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 64; ++j) { mg = fmaxf(mg, fabsf(g[j])); mu = fmaxf(mu, fabsf(u[j])); }
+                    track_g += mg;
+                    track_u += mu;
+                }
             }
             if (!ok) break;
             // h = silu(g) u in fp32, its square summed in fp64, and a bound of what the fp32 pipeline may have lost
@@ -336,13 +350,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
             }
 #endif
             const float cg = eps * P.gnorm[ch], cu = eps * P.unorm[ch];
+            // chunk additions: 2^-24 of every running sum's magnitude, TC_TRACK * (samples + |x| |w|) in all (the
+            // second part is inside eps)
+            const float ag = (float)TC_TRACK * TC_ADD_ULP * track_g * 1.0001f, au = (float)TC_TRACK * TC_ADD_ULP * track_u * 1.0001f;
             const float* xn = P.xnorm + tt * TC_BN + half * 64;
             double e2 = 0.0;
             float eb = 0.f;
 #pragma unroll
             for (int j = 0; j < 64; ++j) {
                 const float at = __ldg(xn + j);
-                const float dg = at * cg, du = at * cu;                 // |g - exact|, |u - exact| at most these
+                const float dg = at * cg + ag, du = at * cu + au;       // |g - exact|, |u - exact| at most these
                 const float gj = g[j], uj = u[j];
                 const float e = __expf(-fmaxf(gj, -80.f));
                 const float s = gj * __fdividef(1.f, 1.f + e);          // silu(g)
@@ -525,7 +542,9 @@ __global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* 
 // rescore_finish_kernel adds the groups in order.
 // Does nothing when the list is empty or longer than max_list (then the full fp64 pass runs instead).
 // ---------------------------------------------------------------------------------------------
-constexpr int RS_CH = 8, RS_TOK = 32, RS_WARPS = 4;
+constexpr int RS_CH = 8, RS_WARPS = 4;
+constexpr int RS_TOK_MIN = 16;             // token groups of the shortest items (part[] is sized for them)
+constexpr int RS_SHORT_LIST = 256;         // lists up to this length use 16-token items (more, shorter items)
 
 __device__ __forceinline__ void dmma_884(double& c0, double& c1, double a, double b) {
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
@@ -538,94 +557,116 @@ __device__ __forceinline__ double bf16x8_elem(const uint4& v, int s) {
     return (double)__uint_as_float((s & 1) ? (w & 0xffff0000u) : (w << 16));
 }
 
+// One warp item: NA A fragments (8 NA tokens from t0) x the 8 listed channels of group grp.
+template <int NA>
+__device__ __forceinline__ void rescore_item(const __nv_bfloat16* __restrict__ X, int L, int d,
+                                             const __nv_bfloat16* __restrict__ Wg, const __nv_bfloat16* __restrict__ Wu,
+                                             const int32_t* __restrict__ list, int n, int grp, int t0, int lane,
+                                             double& e0, double& e1) {
+    const int r = lane >> 2, c = lane & 3;
+    const int nkb = (d + 31) >> 5;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    const __nv_bfloat16* xr[NA];
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+        const int t = t0 + a * 8 + r;
+        xr[a] = t < L ? X + (size_t)t * d + 8 * c : nullptr;
+    }
+    const int li = grp * RS_CH + r;
+    const int ch = li < n ? list[li] : -1;
+    const __nv_bfloat16* wg = ch >= 0 ? Wg + (size_t)ch * d + 8 * c : nullptr;
+    const __nv_bfloat16* wu = ch >= 0 ? Wu + (size_t)ch * d + 8 * c : nullptr;
+    double g[NA][2], u[NA][2];
+#pragma unroll
+    for (int a = 0; a < NA; ++a) { g[a][0] = g[a][1] = u[a][0] = u[a][1] = 0.0; }
+    uint4 vx[NA], vg, vu;
+    auto fetch = [&](int kb) {
+        const bool in = (kb << 5) + 8 * c < d;          // d is a multiple of 8: a vector is inside or outside
+#pragma unroll
+        for (int a = 0; a < NA; ++a) vx[a] = (xr[a] && in) ? __ldg(reinterpret_cast<const uint4*>(xr[a] + (kb << 5))) : zero;
+        vg = (wg && in) ? __ldg(reinterpret_cast<const uint4*>(wg + (kb << 5))) : zero;
+        vu = (wu && in) ? __ldg(reinterpret_cast<const uint4*>(wu + (kb << 5))) : zero;
+    };
+    fetch(0);
+    for (int kb = 0; kb < nkb; ++kb) {
+        uint4 cx[NA];
+#pragma unroll
+        for (int a = 0; a < NA; ++a) cx[a] = vx[a];
+        const uint4 cg = vg, cu = vu;
+        if (kb + 1 < nkb) fetch(kb + 1);                // the next block's loads fly during this block's arithmetic
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+            const double gb = bf16x8_elem(cg, s), ub = bf16x8_elem(cu, s);
+#pragma unroll
+            for (int a = 0; a < NA; ++a) {
+                const double xa = bf16x8_elem(cx[a], s);
+                dmma_884(g[a][0], g[a][1], xa, gb);
+                dmma_884(u[a][0], u[a][1], xa, ub);
+            }
+        }
+    }
+    // lane (r, c) holds token row r of each fragment at listed channels 2c, 2c + 1 of the group; tokens past L gave 0.
+    // Token sum: the fragments in the lane, then the 8 token rows (lanes r = 0..7 of the same c) by shuffles.
+    e0 = 0.0; e1 = 0.0;
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+        const double h0 = silu_f64(g[a][0]) * u[a][0], h1 = silu_f64(g[a][1]) * u[a][1];
+        e0 = fma(h0, h0, e0);
+        e1 = fma(h1, h1, e1);
+    }
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+        e0 += __shfl_xor_sync(0xffffffffu, e0, off);
+        e1 += __shfl_xor_sync(0xffffffffu, e1, off);
+    }
+}
+
+// part is [listed channel][n_tb] with n_tb = ceil(L / RS_TOK_MIN); items of 32 tokens fill every second entry and
+// leave the other zero, so that rescore_finish_kernel adds n_tb entries either way.
 __global__ void __launch_bounds__(32 * RS_WARPS) rescore_list_kernel(const __nv_bfloat16* __restrict__ X, int L, int d,
                                                                       const __nv_bfloat16* __restrict__ Wg,
                                                                       const __nv_bfloat16* __restrict__ Wu,
                                                                       const int32_t* __restrict__ list,
-                                                                      const int* __restrict__ n_list, int max_list, int n_tg,
+                                                                      const int* __restrict__ n_list, int max_list, int n_tb,
                                                                       double* __restrict__ part) {
     const int n = *n_list;
     if (n <= 0 || n > max_list) return;
     const int lane = threadIdx.x & 31, r = lane >> 2, c = lane & 3;
     const int n_grp = (n + RS_CH - 1) / RS_CH;
+    const bool short_items = n <= RS_SHORT_LIST;
+    const int n_tg = short_items ? n_tb : (n_tb + 1) / 2;
     const int items = n_grp * n_tg;
-    const int nkb = (d + 31) >> 5;
-    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     for (int item = blockIdx.x * RS_WARPS + (threadIdx.x >> 5); item < items; item += gridDim.x * RS_WARPS) {
         const int grp = item / n_tg, tg = item - grp * n_tg;
-        const __nv_bfloat16* xr[4];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-            const int t = tg * RS_TOK + a * 8 + r;
-            xr[a] = t < L ? X + (size_t)t * d + 8 * c : nullptr;
-        }
-        const int li = grp * RS_CH + r;
-        const int ch = li < n ? list[li] : -1;
-        const __nv_bfloat16* wg = ch >= 0 ? Wg + (size_t)ch * d + 8 * c : nullptr;
-        const __nv_bfloat16* wu = ch >= 0 ? Wu + (size_t)ch * d + 8 * c : nullptr;
-        double g[4][2], u[4][2];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) { g[a][0] = g[a][1] = u[a][0] = u[a][1] = 0.0; }
-        uint4 vx[4], vg, vu;
-        auto fetch = [&](int kb) {
-            const bool in = (kb << 5) + 8 * c < d;          // d is a multiple of 8: a vector is inside or outside
-#pragma unroll
-            for (int a = 0; a < 4; ++a) vx[a] = (xr[a] && in) ? __ldg(reinterpret_cast<const uint4*>(xr[a] + (kb << 5))) : zero;
-            vg = (wg && in) ? __ldg(reinterpret_cast<const uint4*>(wg + (kb << 5))) : zero;
-            vu = (wu && in) ? __ldg(reinterpret_cast<const uint4*>(wu + (kb << 5))) : zero;
-        };
-        fetch(0);
-        for (int kb = 0; kb < nkb; ++kb) {
-            uint4 cx[4];
-#pragma unroll
-            for (int a = 0; a < 4; ++a) cx[a] = vx[a];
-            const uint4 cg = vg, cu = vu;
-            if (kb + 1 < nkb) fetch(kb + 1);                // the next block's loads fly during this block's arithmetic
-#pragma unroll
-            for (int s = 0; s < 8; ++s) {
-                const double gb = bf16x8_elem(cg, s), ub = bf16x8_elem(cu, s);
-#pragma unroll
-                for (int a = 0; a < 4; ++a) {
-                    const double xa = bf16x8_elem(cx[a], s);
-                    dmma_884(g[a][0], g[a][1], xa, gb);
-                    dmma_884(u[a][0], u[a][1], xa, ub);
-                }
-            }
-        }
-        // lane (r, c) holds token row r of each fragment at listed channels 2c, 2c + 1 of the group; tokens past L gave 0.
-        // Token sum: the 4 fragments in the lane, then the 8 token rows (lanes r = 0..7 of the same c) by shuffles.
-        double e0 = 0.0, e1 = 0.0;
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-            const double h0 = silu_f64(g[a][0]) * u[a][0], h1 = silu_f64(g[a][1]) * u[a][1];
-            e0 = fma(h0, h0, e0);
-            e1 = fma(h1, h1, e1);
-        }
-#pragma unroll
-        for (int off = 4; off < 32; off <<= 1) {
-            e0 += __shfl_xor_sync(0xffffffffu, e0, off);
-            e1 += __shfl_xor_sync(0xffffffffu, e1, off);
-        }
+        double e0, e1;
+        if (short_items) rescore_item<2>(X, L, d, Wg, Wu, list, n, grp, tg * 16, lane, e0, e1);
+        else rescore_item<4>(X, L, d, Wg, Wu, list, n, grp, tg * 32, lane, e0, e1);
         if (r == 0) {
             const int l0 = grp * RS_CH + 2 * c;
-            if (l0 < n) part[(size_t)l0 * n_tg + tg] = e0;
-            if (l0 + 1 < n) part[(size_t)(l0 + 1) * n_tg + tg] = e1;
+            const int slot = short_items ? tg : 2 * tg;
+            if (l0 < n) part[(size_t)l0 * n_tb + slot] = e0;
+            if (l0 + 1 < n) part[(size_t)(l0 + 1) * n_tb + slot] = e1;
+            if (!short_items && slot + 1 < n_tb) {
+                if (l0 < n) part[(size_t)l0 * n_tb + slot + 1] = 0.0;
+                if (l0 + 1 < n) part[(size_t)(l0 + 1) * n_tb + slot + 1] = 0.0;
+            }
         }
     }
 }
 
 // Scores of the re-scored channels: exact energy = sum of the token groups in order, I_i = sqrt(s2_i) n_i, bound 0.
 // With a list longer than max_list every channel was re-scored by the full fp64 pass, whose token ranges
-// (s2part_full [n_split][N]) are added here in order.  Also clears rank[] for the ranking pass that follows.
+// (s2part_full [n_split][N]) are added here in order.  Also clears the rank entries that the ranking pass that
+// follows recomputes: those of the listed channels, or all of them when every score was replaced.
 __global__ void rescore_finish_kernel(const int32_t* __restrict__ list, const int* __restrict__ n_list, int max_list,
                                       const double* __restrict__ part, int n_tb, const double* __restrict__ s2part_full,
                                       int n_split, const double* __restrict__ norm, int N, double* __restrict__ scores,
                                       double* __restrict__ bounds, int32_t* __restrict__ rank_to_zero) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int n = *n_list;
-    if (i < N) rank_to_zero[i] = 0;
     if (n > max_list) {
         if (i < N) {
+            rank_to_zero[i] = 0;
             double s = 0.0;
             for (int y = 0; y < n_split; ++y) s += s2part_full[(size_t)y * N + i];
             scores[i] = sqrt(s) * norm[i];
@@ -639,6 +680,7 @@ __global__ void rescore_finish_kernel(const int32_t* __restrict__ list, const in
     for (int tb = 0; tb < n_tb; ++tb) s += part[(size_t)i * n_tb + tb];
     scores[ch] = sqrt(s) * norm[ch];
     bounds[ch] = 0.0;
+    rank_to_zero[ch] = 0;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -692,7 +734,7 @@ void pop_prefill_tc_plan(int L, int d, int N, PrefillTcPlan* plan) {
     plan->n_pad = plan->n_ct * TC_BM;
     plan->l_pad = plan->n_tt * TC_BN;
     plan->n_parts = 2 * plan->n_tt;
-    plan->n_tb = (L + RS_TOK - 1) / RS_TOK;         // token groups of the list re-scoring kernel
+    plan->n_tb = (L + RS_TOK_MIN - 1) / RS_TOK_MIN;   // token groups of the list re-scoring kernel
     // without the blocked fp64 pass (hidden sizes that are not a multiple of 16) the list kernel takes any length
     plan->max_list = pop_prefill_s2_gemm_supported(d) ? (N < POP_PREFILL_MAX_LIST ? N : POP_PREFILL_MAX_LIST) : N;
 }
