@@ -51,6 +51,39 @@ typedef struct pop_partition pop_partition_t;
 /* Opaque, library-owned: what a prefill needs from one weight set alone (see pop_weights_prepare). */
 typedef struct pop_weights pop_weights_t;
 
+/*
+ * Process-wide settings (host only; the paper has no counterpart: they choose among the library's kernels).
+ *   decode_kernel   which decode kernel family serves partitions created from now on.  POP_DECODE_AUTO: the
+ *                   streaming kernel for bf16 partitions with d in {2048, 4096, 5120} and at most 1536
+ *                   candidates, the fused persistent kernel or, where that does not fit, the multi-kernel
+ *                   path for everything else; POP_DECODE_FUSED / POP_DECODE_SIMPLE force those two.
+ *   launch_mode     how every later step of the streaming kernel is launched.  Its CTAs wait on one
+ *                   another's results.  POP_LAUNCH_PDL (default): plain launch with programmatic stream
+ *                   serialization, which hides the launch latency between the steps of a decode loop but
+ *                   relies on the device being free enough for all CTAs to be resident at once: use it
+ *                   when the decode stream has the device to itself.  POP_LAUNCH_COOPERATIVE: the driver
+ *                   places all CTAs at once or fails the launch (about 2.4 us per step slower): use it
+ *                   when other streams keep SMs busy.  POP_LAUNCH_PLAIN: plain launch.
+ *   wait_budget_us  how long any single device-side wait of a decode step may last before the step gives
+ *                   up (default 50000).  A step that gives up leaves y undefined and is reported by
+ *                   pop_partition_check as POP_ERR_TIMEOUT; it never hangs.
+ *   slab_cache_bytes  device memory of destroyed partitions that the library keeps for the next partition
+ *                   of the same size (default 1 GiB; 0 = keep nothing, and releases what is held).
+ * pop_release_cached_memory() gives all of that memory back to the driver at once (it calls cudaFree,
+ * which synchronises the device).
+ */
+typedef enum { POP_DECODE_AUTO = 0, POP_DECODE_FUSED = 1, POP_DECODE_SIMPLE = 2 } pop_decode_kernel_t;
+typedef enum { POP_LAUNCH_PDL = 0, POP_LAUNCH_COOPERATIVE = 1, POP_LAUNCH_PLAIN = 2 } pop_launch_mode_t;
+typedef struct {
+    pop_decode_kernel_t decode_kernel;
+    pop_launch_mode_t launch_mode;
+    unsigned int wait_budget_us;
+    unsigned long long slab_cache_bytes;
+} pop_config_t;
+int pop_get_config(pop_config_t* out);
+int pop_set_config(const pop_config_t* in);
+int pop_release_cached_memory(void);
+
 /* ---- library information (host only) ------------------------------------------------------- */
 const char* pop_version(void);
 const char* pop_status_string(int status);
@@ -172,8 +205,8 @@ int pop_partition_check(pop_partition_t* p);
 /*
  * Releases everything the partition owns.  The caller must have synchronised the work that used
  * it.  Its device memory may stay with the library for the next partition of the same size on
- * the same device (at most POP_SLAB_CACHE_MB megabytes in all, environment, default 4096, 0 = none):
- * building a partition per prompt and layer then costs no cudaMalloc / cudaFree.
+ * the same device (at most pop_config_t.slab_cache_bytes in all; pop_release_cached_memory() returns
+ * it): building a partition per prompt and layer then costs no cudaMalloc / cudaFree.
  */
 int pop_partition_destroy(pop_partition_t* p);
 
@@ -195,11 +228,11 @@ int pop_partition_destroy(pop_partition_t* p);
  * One partition serves one stream at a time (its scratch and counters are shared by its steps).
  * Two steps of the same call sequence may differ in the last bit of y: partial sums are added to
  * the fp32 accumulator in the order the SMs deliver them; the mask does not depend on that order.
- * The default kernel for bf16 partitions with d in {2048, 4096, 5120} is launched so that its CTAs
- * may take over SMs from the previous kernel of the stream; callers that keep other streams busy
- * on the same device should set POP_STREAM_LAUNCH=coop (cooperative launch) before the first step:
+ * The default kernel for bf16 partitions with d in {2048, 4096, 5120} and at most 1536 candidates is
+ * launched so that its CTAs may take over SMs from the previous kernel of the stream; callers that
+ * keep other streams busy on the same device should choose POP_LAUNCH_COOPERATIVE (pop_set_config):
  * a step whose CTAs cannot all be resident ends with POP_ERR_TIMEOUT at the next
- * pop_partition_check instead of hanging.
+ * pop_partition_check, after at most pop_config_t.wait_budget_us per wait, instead of hanging.
  * Errors: POP_ERR_INVALID_ARG, POP_ERR_UNSUPPORTED (B too large for the shape), POP_ERR_CUDA.
  */
 int pop_decode_step(pop_partition_t* p, const void* x, int B, int k_candidate,

@@ -95,20 +95,20 @@ struct SlabPlan {
 
 // Freed slabs are kept for the next partition of the same device and size instead of going back to the driver:
 // a serving loop builds one partition per prompt and layer, and cudaMalloc / cudaFree (which synchronises the
-// whole device) would otherwise sit in that path.  The cache holds at most POP_SLAB_CACHE_MB megabytes
-// (environment, read once; default 4096; 0 turns it off); what does not fit is freed at once.  A slab enters
-// the cache only through pop_partition_destroy, whose contract is that the caller has synchronised the work
-// that used it.
+// whole device) would otherwise sit in that path.  The cache holds at most pop_config_t.slab_cache_bytes
+// (default 1 GiB; 0 turns it off); what does not fit is freed at once, and pop_release_cached_memory() gives
+// everything back.  A slab enters the cache only through pop_partition_destroy, whose contract is that the
+// caller has synchronised the work that used it.
 namespace {
 struct CachedSlab { int device; size_t bytes; void* ptr; };
 std::mutex g_slab_mutex;
 std::vector<CachedSlab> g_slabs;
 size_t g_slab_bytes = 0;
 
-size_t slab_cache_limit() {
-    static const size_t limit = (size_t)(getenv("POP_SLAB_CACHE_MB") ? atoll(getenv("POP_SLAB_CACHE_MB")) : 4096) << 20;
-    return limit;
-}
+std::mutex g_config_mutex;
+PopConfig g_config = {POP_DECODE_AUTO, POP_LAUNCH_PDL, 50000u, 1ull << 30};
+
+size_t slab_cache_limit() { return (size_t)pop_config_snapshot().slab_cache_bytes; }
 
 void* slab_take(int device, size_t bytes) {
     std::lock_guard<std::mutex> lock(g_slab_mutex);
@@ -123,19 +123,11 @@ void* slab_take(int device, size_t bytes) {
     return nullptr;
 }
 
-void slab_flush() {                      // gives everything back to the driver (current device must own the slabs freed)
+void slab_flush() {                      // gives everything back to the driver (cudaFree takes a pointer of any device)
     std::lock_guard<std::mutex> lock(g_slab_mutex);
-    int cur = 0;
-    cudaGetDevice(&cur);
-    for (size_t i = 0; i < g_slabs.size();) {
-        if (g_slabs[i].device == cur) {
-            cudaFree(g_slabs[i].ptr);
-            g_slab_bytes -= g_slabs[i].bytes;
-            g_slabs.erase(g_slabs.begin() + (long)i);
-        } else {
-            ++i;
-        }
-    }
+    for (size_t i = 0; i < g_slabs.size(); ++i) cudaFree(g_slabs[i].ptr);
+    g_slabs.clear();
+    g_slab_bytes = 0;
 }
 
 bool slab_keep(int device, size_t bytes, void* ptr) {
@@ -146,6 +138,41 @@ bool slab_keep(int device, size_t bytes, void* ptr) {
     return true;
 }
 }  // namespace
+
+PopConfig pop_config_snapshot() {
+    std::lock_guard<std::mutex> lock(g_config_mutex);
+    return g_config;
+}
+
+extern "C" int pop_get_config(pop_config_t* out) {
+    if (!out) return POP_ERR_INVALID_ARG;
+    const PopConfig c = pop_config_snapshot();
+    out->decode_kernel = (pop_decode_kernel_t)c.decode_kernel;
+    out->launch_mode = (pop_launch_mode_t)c.launch_mode;
+    out->wait_budget_us = c.wait_budget_us;
+    out->slab_cache_bytes = c.slab_cache_bytes;
+    return POP_OK;
+}
+
+extern "C" int pop_set_config(const pop_config_t* in) {
+    if (!in) return POP_ERR_INVALID_ARG;
+    if (in->decode_kernel < POP_DECODE_AUTO || in->decode_kernel > POP_DECODE_SIMPLE) return POP_ERR_INVALID_ARG;
+    if (in->launch_mode < POP_LAUNCH_PDL || in->launch_mode > POP_LAUNCH_PLAIN) return POP_ERR_INVALID_ARG;
+    {
+        std::lock_guard<std::mutex> lock(g_config_mutex);
+        g_config.decode_kernel = in->decode_kernel;
+        g_config.launch_mode = in->launch_mode;
+        g_config.wait_budget_us = in->wait_budget_us;
+        g_config.slab_cache_bytes = in->slab_cache_bytes;
+    }
+    if (in->slab_cache_bytes == 0) slab_flush();
+    return POP_OK;
+}
+
+extern "C" int pop_release_cached_memory(void) {
+    slab_flush();
+    return POP_OK;
+}
 
 static void partition_free(pop_partition* p) {
     if (!p) return;
@@ -173,13 +200,13 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     const DeviceInfo& di = device_info(p->device);
     p->sm_count = di.sm_count; p->coop = di.coop; p->max_smem_optin = di.max_smem_optin;
     const size_t row = (size_t)d * p->es;
-    // POP_DECODE_IMPL (read at every partition creation) picks the decode kernel family.  Unset or "stream": tiled
-    // layout + the dataflow kernel of pop_decode_stream.cu for the bf16 shapes it takes (its one-warp selection holds
-    // up to 1536 candidate keys), row layout + the fused / simple kernels for every other shape; "fused" or "simple":
-    // row layout and those kernels for all shapes.
-    const char* impl = getenv("POP_DECODE_IMPL");
-    const bool want_stream = !impl || !*impl || !strcmp(impl, "stream");
-    p->layout = (want_stream && pop_stream_layout_supported(d, dt) && n_cand <= 1536) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
+    // pop_config_t.decode_kernel (as it stands when the partition is created) picks the decode kernel family.
+    // POP_DECODE_AUTO: tiled layout + the dataflow kernel of pop_decode_stream.cu for the bf16 shapes it takes (its
+    // one-warp selection holds up to 1536 candidate keys), row layout + the fused / simple kernels for every other
+    // shape; POP_DECODE_FUSED / POP_DECODE_SIMPLE: row layout and those kernels for all shapes.
+    const int want = pop_config_snapshot().decode_kernel;
+    p->layout = (want == POP_DECODE_AUTO && pop_stream_layout_supported(d, dt) && n_cand <= 1536) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
+    p->force_simple = want == POP_DECODE_SIMPLE;
     p->n_rt = (n_ret + 7) / 8;
     p->n_cg = (n_ret + 15) / 16;
     p->n_ct = (n_cand + 7) / 8;

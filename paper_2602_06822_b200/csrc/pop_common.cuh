@@ -45,6 +45,7 @@ struct pop_partition {
     int es;                       // element size in bytes
     int n_ret, n_cand, n_pruned, n_rc;
     int layout;                   // POP_LAYOUT_*
+    int force_simple;             // rows layout: use the multi-kernel decode path even where the fused kernel would do
     int n_rt, n_ct, n_cg, n_ret_pad, h_stride;      // tiled layout only (h_stride: both)
 
     void* slab;                   // the one device allocation all pointers below point into
@@ -98,6 +99,15 @@ struct WeightStats {
     const void* map_g;            // encoded tensor maps of Wg / Wu (128 bytes each), or NULL: encode per call
     const void* map_u;
 };
+
+// Process-wide settings (pop_set_config); a snapshot is taken where a decision is made.
+struct PopConfig {
+    int decode_kernel;                    // POP_DECODE_AUTO / _FUSED / _SIMPLE: applies when a partition is created
+    int launch_mode;                      // POP_LAUNCH_*: applies to every later step of the streaming kernel
+    unsigned wait_budget_us;              // how long a device-side wait may last before the step gives up
+    unsigned long long slab_cache_bytes;  // freed partition memory kept for reuse, at most
+};
+PopConfig pop_config_snapshot();
 
 // sync[] word assignment (contended counters sit on separate 128-byte lines)
 enum { SYNC_BARRIER = 0, SYNC_TICKET = 1, SYNC_ERROR = 2, SYNC_WORK = 3,
@@ -230,6 +240,25 @@ template <> struct Elem<__nv_bfloat16> {
 // silu(z) = z / (1 + exp(-z)), in the precision of the argument.
 __device__ __forceinline__ double silu_f64(double z) { return z / (1.0 + exp(-z)); }
 __device__ __forceinline__ float silu_f32(float z) { return z / (1.0f + expf(-z)); }
+
+__device__ __forceinline__ unsigned long long pop_global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Budget of a device-side wait in wall time.  The timer is read only every 64 polls (reading it is not free), so a
+// wait that ends within 64 polls never touches it; with a budget of 0 the wait gives up at the first reading.
+struct PopWaitClock {
+    u32 polls;
+    unsigned long long t0;
+    __device__ __forceinline__ PopWaitClock() : polls(0u), t0(0ull) {}
+    __device__ __forceinline__ bool expired(unsigned long long budget_ns) {
+        if ((++polls & 63u) != 0u) return false;
+        const unsigned long long now = pop_global_ns();
+        if (polls == 64u) { t0 = now; return budget_ns == 0ull; }
+        return now - t0 > budget_ns;
+    }
+};
 
 // Scores are non-negative finite doubles: their bit patterns order like the values.
 __device__ __forceinline__ u64 score_key(double s) { return (u64)__double_as_longlong(s); }

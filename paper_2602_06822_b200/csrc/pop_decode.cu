@@ -30,7 +30,6 @@
 namespace {
 
 constexpr int SEL_NT = 128;                 // selector threads (4 warps)
-constexpr u32 SPIN_LIMIT = 1u << 22;        // polls before a wait gives up (of the order of a second)
 constexpr int STAGE_TARGET = 32 * 1024;     // bytes per ring stage aimed for
 constexpr int KEYS_SMEM_MAX = 4096;         // candidate keys kept in shared memory up to this many
 
@@ -54,6 +53,7 @@ struct DecodeParams {
     int T1, T2r, T2c;
     int ncw, MC, MCC, capr, capc, keys_in_smem;
     int off_x, off_pf, off_pd, off_h2, off_mysel, off_keys, off_selsm, off_bars;
+    unsigned long long wait_ns;    // budget of every device-side wait
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -109,11 +109,12 @@ __device__ __forceinline__ void named_bar(int id, int nthreads) {
 }
 
 // Bounded mbarrier wait.  Returns false (and raises the error flags) when it gives up.
-__device__ __forceinline__ bool mbar_wait(u32 bar, u32 parity, volatile int* abort_flag, u32* gerr, int code) {
-    u32 spins = 0;
+__device__ __forceinline__ bool mbar_wait(u32 bar, u32 parity, volatile int* abort_flag, u32* gerr, int code,
+                                          unsigned long long wait_ns) {
+    PopWaitClock spins;
     while (!mbar_try_wait(bar, parity)) {
         if (*abort_flag) return false;
-        if (++spins > SPIN_LIMIT) {
+        if (spins.expired(wait_ns)) {
             *abort_flag = 1;
             atomicExch(gerr, (u32)code);
             return false;
@@ -123,11 +124,12 @@ __device__ __forceinline__ bool mbar_wait(u32 bar, u32 parity, volatile int* abo
 }
 
 // Bounded wait until *counter >= target (grid barrier).
-__device__ __forceinline__ bool grid_wait(const u32* counter, u32 target, volatile int* abort_flag, u32* gerr) {
-    u32 spins = 0;
+__device__ __forceinline__ bool grid_wait(const u32* counter, u32 target, volatile int* abort_flag, u32* gerr,
+                                          unsigned long long wait_ns) {
+    PopWaitClock spins;
     while (ld_acquire_gpu(counter) < target) {
         if (*abort_flag) return false;
-        if (++spins > SPIN_LIMIT) {
+        if (spins.expired(wait_ns)) {
             *abort_flag = 1;
             atomicExch(gerr, (u32)ERR_GRID_BARRIER);
             return false;
@@ -220,7 +222,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
             bool ok = true;
             for (int i = 0; i < n1 && ok; ++i, ++n) {
                 const int s = n % P.nstage, use = n / P.nstage;
-                ok = mbar_wait(empty0 + 8 * s, (use & 1) ^ 1, abort_flag, gerr, ERR_MBAR_EMPTY);
+                ok = mbar_wait(empty0 + 8 * s, (use & 1) ^ 1, abort_flag, gerr, ERR_MBAR_EMPTY, P.wait_ns);
                 if (!ok) break;
                 const int ch0 = (cta + i * G) * TC;
                 const int nch = min(TC, n_rc - ch0);
@@ -230,7 +232,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
             }
             for (int i = 0; i < n2r && ok; ++i, ++n) {
                 const int s = n % P.nstage, use = n / P.nstage;
-                ok = mbar_wait(empty0 + 8 * s, (use & 1) ^ 1, abort_flag, gerr, ERR_MBAR_EMPTY);
+                ok = mbar_wait(empty0 + 8 * s, (use & 1) ^ 1, abort_flag, gerr, ERR_MBAR_EMPTY, P.wait_ns);
                 if (!ok) break;
                 const int r0 = (j0r + i * G) * TR;
                 const int nr = min(TR, n_ret - r0);
@@ -238,10 +240,10 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
                 mbar_expect_tx(full0 + 8 * s, bytes);
                 bulk_g2s(ring_u + s * P.stage_bytes, P.WdT + (size_t)r0 * P.row_bytes, bytes, full0 + 8 * s, pol);
             }
-            if (n2c > 0 && ok) ok = mbar_wait(selbar, 0, abort_flag, gerr, ERR_SELECT);
+            if (n2c > 0 && ok) ok = mbar_wait(selbar, 0, abort_flag, gerr, ERR_SELECT, P.wait_ns);
             for (int i = 0; i < n2c && ok; ++i, ++n) {
                 const int s = n % P.nstage, use = n / P.nstage;
-                ok = mbar_wait(empty0 + 8 * s, (use & 1) ^ 1, abort_flag, gerr, ERR_MBAR_EMPTY);
+                ok = mbar_wait(empty0 + 8 * s, (use & 1) ^ 1, abort_flag, gerr, ERR_MBAR_EMPTY, P.wait_ns);
                 if (!ok) break;
                 const int p0 = (j0c + i * G) * TR;
                 const int nr = min(TR, P.k - p0);
@@ -256,8 +258,8 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
                 // drain: every stage this thread filled must have landed before the CTA may exit
                 for (int m = max(0, n - P.nstage); m < n; ++m) {
                     const int s = m % P.nstage, use = m / P.nstage;
-                    u32 spins = 0;
-                    while (!mbar_try_wait(full0 + 8 * s, use & 1) && ++spins < SPIN_LIMIT) {}
+                    PopWaitClock spins;
+                    while (!mbar_try_wait(full0 + 8 * s, use & 1) && !spins.expired(P.wait_ns)) {}
                 }
             }
         }
@@ -268,7 +270,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
         if (need) {
             bool ok = true;
             if (P.k > 0) {
-                if (st == 0) ok = grid_wait(P.sync + SYNC_BARRIER, (u32)G, abort_flag, gerr);
+                if (st == 0) ok = grid_wait(P.sync + SYNC_BARRIER, (u32)G, abort_flag, gerr, P.wait_ns);
                 group_sync<SEL_NT>(2);
                 ok = !*abort_flag;
             }
@@ -333,7 +335,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
         const u32 ring_u = smem_u32(ring);
         for (int i = 0; i < n1; ++i, ++n) {
             const int s = n % P.nstage, use = n / P.nstage;
-            if (ok) ok = mbar_wait(full0 + 8 * s, use & 1, abort_flag, gerr, ERR_MBAR_FULL);
+            if (ok) ok = mbar_wait(full0 + 8 * s, use & 1, abort_flag, gerr, ERR_MBAR_FULL, P.wait_ns);
             if (!ok) break;
             const int ch0 = (cta + i * G) * TC;
             const int nch = min(TC, n_rc - ch0);
@@ -447,7 +449,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
         // ------------------------------------------------------------------ grid barrier
         if (tc == 0) {
             atomicAdd(P.sync + SYNC_BARRIER, 1u);
-            grid_wait(P.sync + SYNC_BARRIER, (u32)G, abort_flag, gerr);
+            grid_wait(P.sync + SYNC_BARRIER, (u32)G, abort_flag, gerr, P.wait_ns);
         }
         named_bar(1, NTC);
         ok = ok && !*abort_flag;
@@ -472,7 +474,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
         named_bar(1, NTC);
         for (int i = 0; i < n2r; ++i, ++n) {
             const int s = n % P.nstage, use = n / P.nstage;
-            if (ok) ok = mbar_wait(full0 + 8 * s, use & 1, abort_flag, gerr, ERR_MBAR_FULL);
+            if (ok) ok = mbar_wait(full0 + 8 * s, use & 1, abort_flag, gerr, ERR_MBAR_FULL, P.wait_ns);
             if (!ok) break;
             const int r0 = (j0r + i * G) * TR;
             const int nr = min(TR, n_ret - r0);
@@ -497,7 +499,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
             if (lane == 0) mbar_arrive(empty0 + 8 * s);
         }
         if (n2c > 0) {
-            if (ok) ok = mbar_wait(selbar, 0, abort_flag, gerr, ERR_SELECT);
+            if (ok) ok = mbar_wait(selbar, 0, abort_flag, gerr, ERR_SELECT, P.wait_ns);
             float* h2c = h2 + P.capr * BT;
             if (ok) {
                 for (int idx = tc; idx < n2c * TR * BT; idx += NTC) {
@@ -510,7 +512,7 @@ __global__ void __launch_bounds__(672, 1) pop_decode_fused_kernel(const DecodePa
             named_bar(1, NTC);
             for (int i = 0; i < n2c; ++i, ++n) {
                 const int s = n % P.nstage, use = n / P.nstage;
-                if (ok) ok = mbar_wait(full0 + 8 * s, use & 1, abort_flag, gerr, ERR_MBAR_FULL);
+                if (ok) ok = mbar_wait(full0 + 8 * s, use & 1, abort_flag, gerr, ERR_MBAR_FULL, P.wait_ns);
                 if (!ok) break;
                 const int p0 = (j0c + i * G) * TR;
                 const int nr = min(TR, P.k - p0);
@@ -621,17 +623,13 @@ int pop_launch_decode(pop_partition* p, const void* x, int B, int k, void* y, ui
                       int32_t* sel_out, cudaStream_t st) {
     if (!p->coop || p->n_rc <= 0 || p->n_ret + k <= 0) return POP_ERR_UNSUPPORTED;
     if (B > 2) return POP_ERR_UNSUPPORTED;
-    // tuning knobs (read once): POP_DECODE_IMPL=simple forces the multi-kernel path,
-    // POP_STAGE_BYTES overrides the ring stage size aimed for
-    static const char* impl_env = getenv("POP_DECODE_IMPL");
-    if (impl_env && !strcmp(impl_env, "simple")) return POP_ERR_UNSUPPORTED;
-    static const int stage_target = getenv("POP_STAGE_BYTES") ? atoi(getenv("POP_STAGE_BYTES")) : STAGE_TARGET;
+    if (p->force_simple) return POP_ERR_UNSUPPORTED;
+    const int stage_target = STAGE_TARGET;
     const int BT = B;
     const int es = p->es, d = p->d, VEC = 16 / es;
     const int chunks = (d + 32 * VEC - 1) / (32 * VEC);
     // consumer warps / chunks per warp: least padding, CPW in {1, 2, 4}
-    // tuning knob (read once): preferred number of consumer warps
-    static const int ncw_pref = getenv("POP_FUSED_WARPS") ? atoi(getenv("POP_FUSED_WARPS")) : 16;
+    const int ncw_pref = 16;                                  // preferred number of consumer warps
     const int order[] = {ncw_pref, 8, 10, 12, 16, 6, 7, 9, 11, 5, 4};
     int ncw = 0, CPW = 0, best = 1 << 30;
     for (int o : order) {
@@ -666,6 +664,7 @@ int pop_launch_decode(pop_partition* p, const void* x, int B, int k, void* y, ui
     P.capr = ((P.T2r + G - 1) / G) * P.TR;
     P.capc = ((P.T2c + G - 1) / G) * P.TR;
     P.keys_in_smem = p->n_cand <= KEYS_SMEM_MAX;
+    P.wait_ns = 1000ull * (unsigned long long)pop_config_snapshot().wait_budget_us;
 
     // shared-memory layout after the ring
     int off = 0;

@@ -29,6 +29,15 @@ class Ratios(C.Structure):
     _fields_ = [("retained", C.c_double), ("candidate", C.c_double), ("pruned", C.c_double)]
 
 
+class Config(C.Structure):
+    _fields_ = [("decode_kernel", C.c_int), ("launch_mode", C.c_int), ("wait_budget_us", C.c_uint),
+                ("slab_cache_bytes", C.c_ulonglong)]
+
+
+POP_DECODE_AUTO, POP_DECODE_FUSED, POP_DECODE_SIMPLE = 0, 1, 2
+POP_LAUNCH_PDL, POP_LAUNCH_COOPERATIVE, POP_LAUNCH_PLAIN = 0, 1, 2
+
+
 class PopError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -47,6 +56,9 @@ SIGNATURES = {
     "pop_status_string": (C.c_char_p, [C.c_int]),
     "pop_last_cuda_error": (C.c_char_p, []),
     "pop_kernel_launch_count": (C.c_ulonglong, []),
+    "pop_get_config": (C.c_int, [C.POINTER(Config)]),
+    "pop_set_config": (C.c_int, [C.POINTER(Config)]),
+    "pop_release_cached_memory": (C.c_int, []),
     "pop_region_sizes": (C.c_int, [C.c_int, Ratios] + [C.POINTER(C.c_int)] * 4),
     "pop_prefill_partition": (C.c_int, [_P, C.c_int, C.c_int, _P, _P, _P, C.c_int, C.c_int, Ratios, _P,
                                         C.POINTER(_P)]),
@@ -97,6 +109,29 @@ def status_string(status: int) -> str:
 def _check(status: int, where: str):
     if status != POP_OK:
         raise PopError(status, where)
+
+
+def get_config() -> Config:
+    c = Config()
+    _check(lib().pop_get_config(C.byref(c)), "pop_get_config")
+    return c
+
+
+def set_config(**fields) -> Config:
+    """pop_set_config with the named fields replaced (decode_kernel, launch_mode, wait_budget_us, slab_cache_bytes);
+    returns the settings that were in force before."""
+    old = get_config()
+    new = Config(old.decode_kernel, old.launch_mode, old.wait_budget_us, old.slab_cache_bytes)
+    for k, v in fields.items():
+        if k not in dict(Config._fields_):
+            raise KeyError(k)
+        setattr(new, k, v)
+    _check(lib().pop_set_config(C.byref(new)), "pop_set_config")
+    return old
+
+
+def release_cached_memory():
+    _check(lib().pop_release_cached_memory(), "pop_release_cached_memory")
 
 
 def region_sizes(N: int, ratios) -> Tuple[int, int, int, int]:

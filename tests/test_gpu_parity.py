@@ -20,11 +20,13 @@ def _built():
 
 
 @pytest.fixture(autouse=True, params=["fused", "stream"])
-def decode_impl(request, monkeypatch):
+def decode_impl(request):
     """Every case runs with both decode kernel families (the choice is made when a partition is created;
     shapes the streaming kernel does not take use the fused / simple kernels either way)."""
-    monkeypatch.setenv("POP_DECODE_IMPL", request.param)
-    return request.param
+    old = pop.set_config(decode_kernel=pop.POP_DECODE_FUSED if request.param == "fused" else pop.POP_DECODE_AUTO)
+    yield request.param
+    pop.set_config(decode_kernel=old.decode_kernel, launch_mode=old.launch_mode, wait_budget_us=old.wait_budget_us,
+                   slab_cache_bytes=old.slab_cache_bytes)
 
 
 def weights_dev(w):
@@ -369,43 +371,94 @@ def test_all_candidate_scores_equal(d, dtype):
     part.destroy()
 
 
-_LAUNCH_MODE_SCRIPT = r"""
-import sys
-import numpy as np, torch
-sys.path.insert(0, {root!r})
-from oracle import pop_oracle as po
-from paper_2602_06822_b200 import pop, workloads as wl
-from tests import parity as pr
-cfg = wl.FFNConfig("modes", d=2048, N=1536, dtype=wl.BF16, prompt_tokens=24, decode_steps=3,
-                   ratios=wl.Ratios(0.5, 0.25, 0.25), seed=11)
-w = wl.make_ffn_workload(cfg)
-Wh = tuple(np.asarray(a.values, dtype=np.float64) for a in (w.weights.Wg, w.weights.Wu, w.weights.Wd))
-Wg, Wu, Wd = (pr.to_dev(a) for a in (w.weights.Wg, w.weights.Wu, w.weights.Wd))
-part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, cfg.ratios.astuple())
-part.streamed_scores()          # raises unless the streaming kernel serves this partition
-R, C, _ = part.indices()
-k = part.n_cand // 2
-mask = torch.zeros(part.n_cand, dtype=torch.uint8, device="cuda:0")
-for t in range(3):
-    y = pop.decode_step(part, pr.to_dev(w.xs, index=t), k, mask_out=mask)
-    torch.cuda.synchronize()
-    part.check()
-    o = po.decode_step(w.xs.values[t], *Wh, R, C, k)
-    assert np.array_equal(mask.cpu().numpy(), o["mask"])
-    assert pr.rel_err(pr.host_values(y), o["y"]) <= pr.TOL[wl.BF16]
-print("mode ok")
-"""
+def _stream_case():
+    cfg = wl.FFNConfig("modes", d=2048, N=1536, dtype=wl.BF16, prompt_tokens=24, decode_steps=3,
+                       ratios=wl.Ratios(0.5, 0.25, 0.25), seed=11)
+    w = wl.make_ffn_workload(cfg)
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, cfg.ratios.astuple())
+    part.streamed_scores()          # raises unless the streaming kernel serves this partition
+    return w, Wh, part
 
 
-@pytest.mark.gpu
+def _check_steps(w, Wh, part, steps):
+    R, C, _ = part.indices()
+    k = part.n_cand // 2
+    mask = torch.zeros(part.n_cand, dtype=torch.uint8, device="cuda:0")
+    for t in range(steps):
+        y = pop.decode_step(part, pr.to_dev(w.xs, index=t), k, mask_out=mask)
+        torch.cuda.synchronize()
+        part.check()
+        o = po.decode_step(w.xs.values[t], *Wh, R, C, k)
+        assert np.array_equal(mask.cpu().numpy(), o["mask"])
+        assert pr.rel_err(pr.host_values(y), o["y"]) <= pr.TOL[wl.BF16]
+
+
 @pytest.mark.parametrize("mode", ["pdl", "coop", "plain"])
 def test_streaming_kernel_launch_modes(mode, decode_impl):
-    """The launch mode of the streaming kernel is read once per process, so each mode runs in a process of its own."""
+    """The launch mode is a process-wide setting read at every step: the same partition is stepped in each mode."""
     if decode_impl != "stream":
         pytest.skip("launch modes belong to the streaming kernel")
-    import os, subprocess, sys
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    env = dict(os.environ, POP_STREAM_LAUNCH=mode, POP_DECODE_IMPL="stream")
-    out = subprocess.run([sys.executable, "-c", _LAUNCH_MODE_SCRIPT.format(root=root)], env=env, cwd=root,
-                         capture_output=True, text=True, timeout=600)
-    assert out.returncode == 0 and "mode ok" in out.stdout, out.stdout[-2000:] + out.stderr[-2000:]
+    w, Wh, part = _stream_case()
+    code = {"pdl": pop.POP_LAUNCH_PDL, "coop": pop.POP_LAUNCH_COOPERATIVE, "plain": pop.POP_LAUNCH_PLAIN}[mode]
+    old = pop.set_config(launch_mode=code)
+    try:
+        assert pop.get_config().launch_mode == code
+        _check_steps(w, Wh, part, 3)
+    finally:
+        pop.set_config(launch_mode=old.launch_mode)
+    part.destroy()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_partition_stays_usable(decode_impl):
+    """Failure detection without a fault: with a wait budget of zero every device-side wait that is not satisfied
+    within its first polls gives up, the step winds down (all CTAs drain and leave), pop_partition_check reports
+    POP_ERR_TIMEOUT, and with the budget restored the next steps on the same partition are correct again."""
+    if decode_impl != "stream":
+        pytest.skip("the streaming kernel is the one whose CTAs wait on one another")
+    w, Wh, part = _stream_case()
+    old = pop.set_config(wait_budget_us=0)
+    try:
+        timed_out = 0
+        for t in range(3):
+            pop.decode_step(part, pr.to_dev(w.xs, index=t), part.n_cand // 2)
+            try:
+                part.check()
+            except pop.PopError as e:
+                assert e.status == pop.POP_ERR_TIMEOUT
+                timed_out += 1
+    finally:
+        pop.set_config(wait_budget_us=old.wait_budget_us)
+    assert timed_out > 0, "no wait ran out with a zero budget"
+    _check_steps(w, Wh, part, 3)
+    part.destroy()
+
+
+def test_config_rejects_bad_values_and_cache_can_be_released():
+    c = pop.get_config()
+    for bad in ({"decode_kernel": 7}, {"launch_mode": -1}):
+        with pytest.raises(pop.PopError) as e:
+            pop.set_config(**bad)
+        assert e.value.status == pop.POP_ERR_INVALID_ARG
+    assert pop.get_config().launch_mode == c.launch_mode
+    pop.release_cached_memory()
+
+
+@pytest.mark.parametrize("d,N,L,dtype", [(512, 1500, 70, wl.BF16), (2048, 900, 40, wl.BF16), (264, 777, 33, wl.F32)])
+def test_prepared_weights_give_the_same_partition(d, N, L, dtype):
+    """pop_weights_prepare + pop_prefill_partition_prepared against pop_prefill_partition: same regions and scores, bit
+    for bit, for two prompts on one prepared weight set."""
+    cfg = wl.FFNConfig("prep", d=d, N=N, dtype=dtype, prompt_tokens=L, decode_steps=1, ratios=wl.Ratios(0.5, 0.2, 0.3), seed=41)
+    w = wl.make_ffn_workload(cfg)
+    Wg, Wu, Wd = weights_dev(w)
+    wts = pop.Weights(Wg, Wu, Wd)
+    X = pr.to_dev(w.X)
+    for Xi in (X, X[: L // 2].contiguous()):
+        a = pop.prefill_partition(Xi, Wg, Wu, Wd, cfg.ratios.astuple())
+        b = wts.prefill_partition(Xi, cfg.ratios.astuple())
+        for ia, ib in zip(a.indices(), b.indices()):
+            assert np.array_equal(ia, ib)
+        assert np.array_equal(a.scores(), b.scores()) and np.array_equal(a.score_bounds(), b.score_bounds())
+        a.destroy(); b.destroy()
+    wts.destroy()
