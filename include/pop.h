@@ -148,6 +148,22 @@ int pop_prefill_partition_prepared(const void* X, int L, const pop_weights_t* w,
 int pop_weights_destroy(pop_weights_t* w);
 
 /*
+ * The prefilling stage together with the prompt's own block output "under the resulting pruning structure"
+ * (Sec. 3.4).  The paper does not say which channels that structure keeps for the prompt; the reading taken
+ * here is the mask a static variant would reuse at every step (Sec. 4.6, Variant (1)): Retained plus the
+ * k_candidate Candidates with the largest PREFILL score (ties by lower channel id), i.e. the n_ret + k_candidate
+ * best channels by I_i.
+ *   Y [L, d]: device array of the weights' dtype, caller-owned:
+ *   Y[t] = sum over those channels i of Wd[:, i] * silu(Wg[i].X[t]) * (Wu[i].X[t]).
+ * Everything else as pop_prefill_partition_prepared.  The intermediate activations of the scoring pass (fp32
+ * accumulation on the tensor cores) are kept as bf16 pairs (16 significant bits) and contracted with Wd by a second tensor-core pass (fp32
+ * accumulation, one rounding to bf16 at the end); the mask itself is decided on exact scores like the regions.
+ * bf16 with d >= 64 and N a multiple of 8 only (POP_ERR_UNSUPPORTED otherwise); 0 <= k_candidate <= n_cand.
+ */
+int pop_prefill_partition_with_output(const void* X, int L, const pop_weights_t* w, pop_ratios_t ratios,
+                                      int k_candidate, void* Y, void* cuda_stream, pop_partition_t** out);
+
+/*
  * Build a partition from caller-chosen regions instead of prefill scores (the regions of
  * Sec. 3.3 given explicitly).  h_ret [n_ret] and h_cand [n_cand] are HOST arrays of channel
  * ids, each strictly ascending, disjoint, in [0, N); channels in neither are Pruned.

@@ -319,10 +319,15 @@ extern "C" int pop_weights_destroy(pop_weights_t* w) {
 // are computed into this call's temporaries.
 static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, const void* Wu, const void* Wd, int N,
                                   pop_dtype_t dtype, pop_ratios_t ratios, const pop_weights* prepared, cudaStream_t st,
-                                  pop_partition_t** out) {
+                                  pop_partition_t** out, int k_out = -1, void* Y = nullptr) {
     int n_ret, n_cand, n_pruned;
     int rc = pop_region_sizes(N, ratios, &n_ret, &n_cand, &n_pruned, nullptr);
     if (rc != POP_OK) return rc;
+    const bool want_y = Y != nullptr;
+    if (want_y) {
+        if (k_out < 0 || k_out > n_cand) return POP_ERR_INVALID_ARG;
+        if (!pop_prefill_output_supported(d, N, dtype)) return POP_ERR_UNSUPPORTED;
+    }
     pop_partition* p = nullptr;
     rc = partition_alloc(d, N, dtype, n_ret, n_cand, st, &p);
     if (rc != POP_OK) return rc;
@@ -337,8 +342,9 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
     const size_t t_norm = tmp.take(prepared ? 0 : sizeof(double) * (size_t)N);
     const size_t t_s2 = tmp.take(tc ? 0 : sizeof(double) * (size_t)N);
     const size_t t_s2part = tmp.take(gemm ? sizeof(double) * (size_t)N * (size_t)pop_prefill_s2_gemm_splits(L) : 0);
-    size_t t_xn = 0, t_gn = 0, t_un = 0, t_tp = 0, t_bp = 0, t_mm = 0, t_list = 0, t_nl = 0, t_part = 0;
+    size_t t_xn = 0, t_gn = 0, t_un = 0, t_tp = 0, t_bp = 0, t_mm = 0, t_list = 0, t_nl = 0, t_part = 0, t_H = 0;
     if (tc) {
+        t_H = tmp.take(want_y ? sizeof(__nv_bfloat16) * 2 * (size_t)tp.l_pad * tp.n_pad : 0);
         t_xn = tmp.take(sizeof(float) * (size_t)tp.l_pad);
         t_gn = tmp.take(prepared ? 0 : sizeof(float) * (size_t)tp.n_pad);
         t_un = tmp.take(prepared ? 0 : sizeof(float) * (size_t)tp.n_pad);
@@ -371,13 +377,15 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
     PrefillTcScratch sc;
     if (rc == POP_OK && tc) {
         sc.xnorm = (float*)(tb + t_xn); sc.gnorm = nullptr; sc.unorm = nullptr;
+        sc.H = want_y ? (void*)(tb + t_H) : nullptr;
         sc.s2part = (double*)(tb + t_tp); sc.bpart = (float*)(tb + t_bp); sc.m_max = (u64*)(tb + t_mm);
         sc.list = (int32_t*)(tb + t_list); sc.n_list = (int*)(tb + t_nl); sc.part = (double*)(tb + t_part);
         sc.rank = p->rank_tmp;
         sc.s2part_full = s2part;
         rc = pop_launch_prefill_tc(X, L, d, Wg, Wu, N, ws, sc, p->scores, p->score_bounds, p->sync + SYNC_ERROR, p->sm_count, st);
         if (rc == POP_OK)
-            rc = pop_launch_prefill_rescore(X, L, d, Wg, Wu, N, ws.norm, n_ret, n_cand, sc, p->scores, p->score_bounds, p->sm_count, st);
+            rc = pop_launch_prefill_rescore(X, L, d, Wg, Wu, N, ws.norm, n_ret, n_cand, want_y ? n_ret + k_out : 0, sc, p->scores,
+                                            p->score_bounds, p->sm_count, st);
     } else if (rc == POP_OK) {
         double* s2 = (double*)(tb + t_s2);
         rc = gemm ? pop_launch_prefill_s2_gemm(X, L, d, Wg, Wu, N, dtype, s2part, s2, st)
@@ -391,10 +399,25 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
                 : pop_launch_partition(p->scores, N, n_ret, n_cand, p->rank_tmp, p->sm_count, p->idx_ret, p->idx_cand, p->idx_pruned, st);
     if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, ws.norm, st)
                                                          : pop_launch_repack(p, Wg, Wu, Wd, ws.norm, st);
+    // the prompt's own output under the mask rank < n_ret + k (the ranks are final for every channel near that boundary)
+    if (rc == POP_OK && want_y)
+        rc = pop_launch_prefill_output(sc.H, L, d, Wd, N, p->rank_tmp, n_ret + k_out, Y, p->sync + SYNC_ERROR, p->sm_count, st);
     cudaFreeAsync(tb, st);
     if (rc != POP_OK) { partition_free_now(p, st); return rc; }
     *out = p;
     return POP_OK;
+}
+
+extern "C" int pop_prefill_partition_with_output(const void* X, int L, const pop_weights_t* w, pop_ratios_t ratios,
+                                                 int k_candidate, void* Y, void* cuda_stream, pop_partition_t** out) {
+    if (!out) return POP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!X || !w || !Y || L <= 0 || !aligned16(X) || !aligned16(Y)) return POP_ERR_INVALID_ARG;
+    int dev = -1;
+    POP_CUDA(cudaGetDevice(&dev));
+    if (dev != w->device) return POP_ERR_INVALID_ARG;
+    return prefill_partition_impl(X, L, w->d, w->Wg, w->Wu, w->Wd, w->N, w->dtype, ratios, w, (cudaStream_t)cuda_stream, out,
+                                  k_candidate, Y);
 }
 
 extern "C" int pop_prefill_partition(const void* X, int L, int d, const void* Wg, const void* Wu, const void* Wd,

@@ -176,6 +176,7 @@ int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* 
 #define POP_PREFILL_MAX_LIST 4096     // longest list the list re-scoring kernel takes; longer lists use the full fp64 pass
 struct PrefillTcPlan { int n_ct, n_tt, n_pad, l_pad, n_parts, n_tb, max_list; };
 struct PrefillTcScratch {
+    void* H;               // [2][l_pad][n_pad] bf16 (high, low) intermediate activations of the prompt, or NULL
     float* xnorm;          // [l_pad]
     float* gnorm;          // [n_pad]
     float* unorm;          // [n_pad]
@@ -197,8 +198,12 @@ int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const voi
                           const PrefillTcScratch& s, double* scores, double* bounds, u32* status, int sm_count,
                           cudaStream_t st);
 int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
-                               int n_ret, int n_cand, const PrefillTcScratch& s, double* scores, double* bounds,
-                               int sm_count, cudaStream_t st);
+                               int n_ret, int n_cand, int n_third /*extra rank boundary, 0 = none*/, const PrefillTcScratch& s,
+                               double* scores, double* bounds, int sm_count, cudaStream_t st);
+// the prompt's own output from H (cleared outside the mask rank < n_active) and Wd [d, N], on the tensor cores
+bool pop_prefill_output_supported(int d, int N, pop_dtype_t dt);
+int pop_launch_prefill_output(void* H, int L, int d, const void* Wd, int N, const int32_t* rank, int n_active, void* Y,
+                              u32* status, int sm_count, cudaStream_t st);
 // pop_decode_stream.cu (bf16 partitions in the tiled layout)
 bool pop_stream_layout_supported(int d, pop_dtype_t dt);
 int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void* y,

@@ -173,6 +173,8 @@ struct TcParams {
     const float* xnorm;           // [n_tt * 128]  |X[t]|_2, rounded up; 0 past L
     const float* gnorm;           // [n_pad]       |Wg[i]|_2, rounded up; 0 past N
     const float* unorm;           // [n_pad]
+    __nv_bfloat16* H;             // [2][n_tt * 128][n_pad] intermediate activations silu(g) u as a bf16 pair (nearest bf16, then
+                                  // nearest bf16 of the remainder: 16 significant bits), or NULL when nobody needs them
     double* s2part;               // [2 n_tt][n_pad] partial energies (token half h of token tile tt at 2 tt + h)
     float* bpart;                 // [2 n_tt][n_pad] bounds of their errors
     u32* status;
@@ -356,6 +358,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
             const float* xn = P.xnorm + tt * TC_BN + half * 64;
             double e2 = 0.0;
             float eb = 0.f;
+            __nv_bfloat16* hrow = P.H ? P.H + (size_t)(tt * TC_BN + half * 64) * P.n_pad + ch : nullptr;
+            const size_t h_lo_off = (size_t)P.n_tt * TC_BN * P.n_pad;
 #pragma unroll
             for (int j = 0; j < 64; ++j) {
                 const float at = __ldg(xn + j);
@@ -370,6 +374,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
                 const float dh = 1.1f * dg * fabsf(uj) + (fabsf(s) + 1.1f * dg) * du + rho * fabsf(h) + 2e-35f * fabsf(gj * uj);
                 eb += 2.f * fabsf(h) * dh + dh * dh;
                 e2 = fma((double)h, (double)h, e2);
+                if (hrow) {                                              // a warp writes 64 contiguous bytes per token and part
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(h);
+                    hrow[(size_t)j * P.n_pad] = hi;
+                    hrow[h_lo_off + (size_t)j * P.n_pad] = __float2bfloat16_rn(h - __bfloat162float(hi));
+                }
             }
             const size_t slot = (size_t)(2 * tt + half) * P.n_pad + ch;
             P.s2part[slot] = e2;
@@ -478,54 +487,60 @@ constexpr int SEL_NT = 1024;
 __global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* __restrict__ scores,
                                                                   const double* __restrict__ bounds,
                                                                   const int32_t* __restrict__ rank, int N, int n_ret, int n_cand,
-                                                                  const u64* __restrict__ m_max, int32_t* __restrict__ list,
-                                                                  int* __restrict__ n_list) {
+                                                                  int n_third, const u64* __restrict__ m_max,
+                                                                  int32_t* __restrict__ list, int* __restrict__ n_list) {
     __shared__ u32 sm[POP_SELECT_SMEM_WORDS(SEL_NT)];
-    __shared__ u64 mw_bits[2];
-    __shared__ double tau_sm[2];
+    __shared__ u64 mw_bits[3];
+    __shared__ double tau_sm[3];
     const int tid = threadIdx.x;
     const double m = __longlong_as_double((long long)*m_max);
     if (!(m > 0.0)) { if (tid == 0) *n_list = 0; return; }
-    const int n1 = n_ret, n2 = n_ret + n_cand;
-    const bool b1 = n1 > 0 && n1 < N, b2 = n2 > 0 && n2 < N && n2 != n1;
+    // rank boundaries: Retained | Candidate, Candidate | Pruned and, when the caller wants the prompt's own output,
+    // the boundary of its mask inside the Candidate region (n_third = n_ret + k; 0 = none)
+    const int n1 = n_ret, n2 = n_ret + n_cand, n3 = n_third;
+    const bool b1 = n1 > 0 && n1 < N, b2 = n2 > 0 && n2 < N && n2 != n1, b3 = n3 > 0 && n3 < N && n3 != n1 && n3 != n2;
     const int per = (N + SEL_NT - 1) / SEL_NT;
     const int lo = min(N, tid * per), hi = min(N, lo + per);
-    if (tid < 2) { mw_bits[tid] = 0ull; tau_sm[tid] = 0.0; }
+    if (tid < 3) { mw_bits[tid] = 0ull; tau_sm[tid] = 0.0; }
     __syncthreads();
     // tau = the streamed score of the channel at rank n - 1 (exactly one channel holds each rank)
     for (int i = lo; i < hi; ++i) {
         const int r = rank[i];
         if (b1 && r == n1 - 1) tau_sm[0] = scores[i];
         if (b2 && r == n2 - 1) tau_sm[1] = scores[i];
+        if (b3 && r == n3 - 1) tau_sm[2] = scores[i];
     }
     __syncthreads();
-    const double tau1 = tau_sm[0], tau2 = tau_sm[1];
+    const double tau1 = tau_sm[0], tau2 = tau_sm[1], tau3 = tau_sm[2];
     // Outside tau +- 2m every channel is placed (argument above).  Inside, the test can use the channel's own bound:
     // with m_W the largest bound inside that window, at most n - 1 channels have a_j + m_j > tau + m_W and at least
     // n have a_j - m_j >= tau - m_W, so a_i - m_i > tau + m_W places i inside the top n and a_i + m_i < tau - m_W
     // outside, by the same two counts.
     const double w = 2.0 * m * (1.0 + 1e-9);
-    double mw1 = 0.0, mw2 = 0.0;
+    double mw1 = 0.0, mw2 = 0.0, mw3 = 0.0;
     for (int i = lo; i < hi; ++i) {
         const double a = scores[i], mi = bounds[i];
         if (b1 && fabs(a - tau1) <= w) mw1 = fmax(mw1, mi);
         if (b2 && fabs(a - tau2) <= w) mw2 = fmax(mw2, mi);
+        if (b3 && fabs(a - tau3) <= w) mw3 = fmax(mw3, mi);
     }
     if (mw1 > 0.0) atomicMax(&mw_bits[0], (u64)__double_as_longlong(mw1));
     if (mw2 > 0.0) atomicMax(&mw_bits[1], (u64)__double_as_longlong(mw2));
+    if (mw3 > 0.0) atomicMax(&mw_bits[2], (u64)__double_as_longlong(mw3));
     __syncthreads();
     mw1 = __longlong_as_double((long long)mw_bits[0]) * (1.0 + 1e-9);
     mw2 = __longlong_as_double((long long)mw_bits[1]) * (1.0 + 1e-9);
+    mw3 = __longlong_as_double((long long)mw_bits[2]) * (1.0 + 1e-9);
+    auto open_at = [&](double a, double mi) -> bool {
+        return (b1 && fabs(a - tau1) <= w && fabs(a - tau1) <= mi + mw1) || (b2 && fabs(a - tau2) <= w && fabs(a - tau2) <= mi + mw2) ||
+               (b3 && fabs(a - tau3) <= w && fabs(a - tau3) <= mi + mw3);
+    };
     int cnt = 0;
-    for (int i = lo; i < hi; ++i) {
-        const double a = scores[i], mi = bounds[i];
-        cnt += (b1 && fabs(a - tau1) <= w && fabs(a - tau1) <= mi + mw1) || (b2 && fabs(a - tau2) <= w && fabs(a - tau2) <= mi + mw2);
-    }
+    for (int i = lo; i < hi; ++i) cnt += open_at(scores[i], bounds[i]);
     int tot;
     int pos = group_excl_scan<SEL_NT>(cnt, sm, tid, 0, tot);
     for (int i = lo; i < hi; ++i) {
-        const double a = scores[i], mi = bounds[i];
-        if ((b1 && fabs(a - tau1) <= w && fabs(a - tau1) <= mi + mw1) || (b2 && fabs(a - tau2) <= w && fabs(a - tau2) <= mi + mw2)) list[pos++] = i;
+        if (open_at(scores[i], bounds[i])) list[pos++] = i;
     }
     if (tid == 0) *n_list = tot;
 }
@@ -683,6 +698,191 @@ __global__ void rescore_finish_kernel(const int32_t* __restrict__ list, const in
     rank_to_zero[ch] = 0;
 }
 
+// ---------------------------------------------------------------------------------------------
+// The prompt's own output under the pruned structure (Sec. 3.4: "the prefilling pass is then completed under the
+// resulting pruning structure"): Y[t, :] = sum over the active channels i of Wd[:, i] H[t, i], the active channels
+// being Retained plus the k best Candidates by prefill score.  H comes from the scoring pass as a bf16 pair
+// (high part + low part: a single bf16 would leave 2^-9 of every term, too much for outputs that nearly cancel); the
+// channels outside the mask are cleared in H (mask_h_kernel), so that the contraction can run over all N channels on
+// plain K-major operands: A = H_hi and H_lo [tokens, N], B = Wd [d, N], all as they lie in memory, no gather.  Both
+// parts of a K slab are multiplied with the same Wd tile.
+// Unit: 128 tokens x 128 outputs over all channels; accumulator in tensor memory (two sets take turns over the
+// units); warp 0 TMA producer, warp 1 MMA issue, warps 2..5 epilogue (warp w reads lanes 32 (w % 4) ..).
+// ---------------------------------------------------------------------------------------------
+constexpr int DN_STAGES = 4;
+constexpr int DN_STAGE_BYTES = 3 * TC_TILE_BYTES;        // H_hi, H_lo, Wd
+constexpr int DN_THREADS = 192;
+constexpr size_t DN_SMEM_BYTES = (size_t)DN_STAGES * DN_STAGE_BYTES + 1024 + 256;
+enum { DN_ERR_PRODUCER = 111, DN_ERR_MMA_FULL = 112, DN_ERR_MMA_ACC = 113, DN_ERR_EPILOGUE = 114 };
+
+struct DownParams {
+    int L, d, n_tt, n_jt, nk;
+    int lo_row;                   // first row of the low parts in the H tensor map
+    __nv_bfloat16* Y;             // [L, d]
+    u32* status;
+};
+
+__global__ void __launch_bounds__(DN_THREADS, 1) prefill_down_kernel(const __grid_constant__ CUtensorMap map_h,
+                                                                     const __grid_constant__ CUtensorMap map_d,
+                                                                     const DownParams P) {
+    extern __shared__ unsigned char dn_smem_raw[];
+    __shared__ u32 tmem_base_slot;
+    __shared__ int abort_flag;
+    const u32 raw = smem_u32(dn_smem_raw);
+    const u32 tiles = (raw + 1023u) & ~1023u;
+    const u32 bars = tiles + DN_STAGES * DN_STAGE_BYTES;
+    const u32 bar_full = bars, bar_empty = bars + 8 * DN_STAGES;
+    const u32 bar_acc_full = bars + 16 * DN_STAGES, bar_acc_empty = bar_acc_full + 16, bar_drain = bar_acc_full + 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abortp = &abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < DN_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_acc_full + 8 * b, 1); mbar_init(bar_acc_empty + 8 * b, 4); }
+        mbar_init(bar_drain, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(256) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const u32 tmem_base = tmem_base_slot;
+    const int n_units = P.n_tt * P.n_jt;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0, issued = 0;
+            u32 ph = 0;
+            bool ok = true;
+            for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+                const int tt = unit / P.n_jt, jt = unit - tt * P.n_jt;
+                for (int kb = 0; kb < P.nk; ++kb) {
+                    ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, abortp, P.status, DN_ERR_PRODUCER);
+                    if (!ok) break;
+                    const u32 dst = tiles + (u32)s * DN_STAGE_BYTES, bar = bar_full + 8 * s;
+                    mbar_expect_tx(bar, DN_STAGE_BYTES);
+                    tma_load_2d(dst, &map_h, kb * TC_BK, tt * 128, bar);
+                    tma_load_2d(dst + TC_TILE_BYTES, &map_h, kb * TC_BK, P.lo_row + tt * 128, bar);
+                    tma_load_2d(dst + 2 * TC_TILE_BYTES, &map_d, kb * TC_BK, jt * 128, bar);
+                    ++issued;
+                    if (++s == DN_STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) {
+                const int back = issued < DN_STAGES ? issued : DN_STAGES;
+                for (int j = 1; j <= back; ++j) {
+                    int sj = s - j;
+                    u32 pj = ph;
+                    if (sj < 0) { sj += DN_STAGES; pj ^= 1u; }
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_full + 8 * sj, pj) && global_ns() - t0 < TC_WAIT_BUDGET_NS) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int s = 0, buf = 0;
+            u32 ph = 0, accph[2] = {0u, 0u};
+            bool ok = true;
+            for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+                ok = mbar_wait(bar_acc_empty + 8 * buf, accph[buf] ^ 1u, abortp, P.status, DN_ERR_MMA_ACC);
+                if (!ok) break;
+                tc_fence_after();
+                const u32 dacc = tmem_base + (u32)buf * 128u;
+                for (int kb = 0; kb < P.nk; ++kb) {
+                    ok = mbar_wait(bar_full + 8 * s, ph, abortp, P.status, DN_ERR_MMA_FULL);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const u32 base = tiles + (u32)s * DN_STAGE_BYTES;
+                    const u64 da = smem_desc_sw128(base), dl = smem_desc_sw128(base + TC_TILE_BYTES),
+                              db = smem_desc_sw128(base + 2 * TC_TILE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k) {
+                        umma_bf16(dacc, da + 2ull * k, db + 2ull * k, TC_IDESC, (kb > 0 || k > 0) ? 1u : 0u);
+                        umma_bf16(dacc, dl + 2ull * k, db + 2ull * k, TC_IDESC, 1u);
+                    }
+                    umma_commit(bar_empty + 8 * s);
+                    if (++s == DN_STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(bar_acc_full + 8 * buf);
+                accph[buf] ^= 1u;
+                buf ^= 1;
+            }
+            umma_commit(bar_drain);
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(bar_drain, 0u) && global_ns() - t0 < TC_WAIT_BUDGET_NS) {}
+        }
+    } else {
+        const int quarter = warp & 3;
+        const u32 lane_base = ((u32)(quarter * 32)) << 16;
+        int buf = 0;
+        u32 accph[2] = {0u, 0u};
+        bool ok = true;
+        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+            const int tt = unit / P.n_jt, jt = unit - tt * P.n_jt;
+            ok = mbar_wait(bar_acc_full + 8 * buf, accph[buf], abortp, P.status, DN_ERR_EPILOGUE);
+            if (!ok) break;
+            tc_fence_after();
+            const int t = tt * 128 + quarter * 32 + lane;
+            const int j0 = jt * 128;
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                float v[32];
+                tmem_ld32(tmem_base + lane_base + (u32)buf * 128u + 32u * p, v);
+                if (t < P.L) {
+                    uint4* dst = reinterpret_cast<uint4*>(P.Y + (size_t)t * P.d + j0 + 32 * p);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        if (j0 + 32 * p + 8 * q < P.d) {                    // d is a multiple of 8
+                            uint4 o;
+                            o.x = (u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 0])) | ((u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 1])) << 16);
+                            o.y = (u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 2])) | ((u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 3])) << 16);
+                            o.z = (u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 4])) | ((u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 5])) << 16);
+                            o.w = (u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 6])) | ((u32)__bfloat16_as_ushort(__float2bfloat16_rn(v[8 * q + 7])) << 16);
+                            dst[q] = o;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
+            accph[buf] ^= 1u;
+            buf ^= 1;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256) : "memory");
+    }
+}
+
+// Clears, in H [rows][n_pad], the columns of the channels outside the prompt's mask: rank[i] >= n_active.
+__global__ void mask_h_kernel(__nv_bfloat16* __restrict__ H, int rows, int n_pad, int N, const int32_t* __restrict__ rank, int n_active) {
+    const int vec_per_row = n_pad >> 3;
+    const size_t total = (size_t)rows * vec_per_row;
+    for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (size_t)gridDim.x * blockDim.x) {
+        const int c0 = (int)(o % vec_per_row) * 8;
+        u32 keep = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) keep |= (c0 + e < N && rank[c0 + e] < n_active) ? (1u << e) : 0u;
+        if (keep == 0xffu) continue;
+        uint4* p = reinterpret_cast<uint4*>(H) + o;
+        uint4 v = *p;
+        u32* w = reinterpret_cast<u32*>(&v);
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if (!((keep >> e) & 1u)) w[e >> 1] &= (e & 1) ? 0x0000ffffu : 0xffff0000u;
+        *p = v;
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -700,12 +900,13 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// [rows, d] bf16 row-major; box = 64 columns (128 bytes, the swizzle span) x 128 rows; out-of-range elements read as zero
-int make_map(CUtensorMap* map, const void* base, int rows, int d) {
+// [rows, d] bf16 row-major (row pitch `pitch` elements); box = 64 columns (128 bytes, the swizzle span) x 128 rows;
+// out-of-range elements read as zero
+int make_map(CUtensorMap* map, const void* base, int rows, int d, int pitch = 0) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) { pop_set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled is not available from this driver"); return POP_ERR_CUDA; }
     const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
+    const cuuint64_t strides[1] = {(cuuint64_t)(pitch ? pitch : d) * 2};
     const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)TC_BM};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
@@ -787,6 +988,7 @@ int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const voi
     P.nk = (d + TC_BK - 1) / TC_BK;
     P.xnorm = s.xnorm; P.gnorm = ws.gnorm; P.unorm = ws.unorm;
     P.s2part = s.s2part; P.bpart = s.bpart; P.status = status;
+    P.H = (__nv_bfloat16*)s.H;
 #ifdef POP_TC_DUMP
     P.dump_g = g_tc_dump_g; P.dump_u = g_tc_dump_u;
 #endif
@@ -802,13 +1004,13 @@ int pop_launch_prefill_tc(const void* X, int L, int d, const void* Wg, const voi
 }
 
 int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, const void* Wu, int N, const double* norm,
-                               int n_ret, int n_cand, const PrefillTcScratch& s, double* scores, double* bounds,
+                               int n_ret, int n_cand, int n_third, const PrefillTcScratch& s, double* scores, double* bounds,
                                int sm_count, cudaStream_t st) {
     PrefillTcPlan plan;
     pop_prefill_tc_plan(L, d, N, &plan);
     const int rc0 = pop_launch_ranks(scores, N, s.rank, sm_count, st);          // s.rank was cleared by tc_finish_kernel
     if (rc0 != POP_OK) return rc0;
-    select_uncertain_kernel<<<1, SEL_NT, 0, st>>>(scores, bounds, s.rank, N, n_ret, n_cand, s.m_max, s.list, s.n_list);
+    select_uncertain_kernel<<<1, SEL_NT, 0, st>>>(scores, bounds, s.rank, N, n_ret, n_cand, n_third, s.m_max, s.list, s.n_list);
     POP_LAUNCHED();
     rescore_list_kernel<<<sm_count * 4, 32 * RS_WARPS, 0, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg,
                                                         (const __nv_bfloat16*)Wu, s.list, s.n_list, plan.max_list,
@@ -821,6 +1023,35 @@ int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, cons
     }
     rescore_finish_kernel<<<(N + 255) / 256, 256, 0, st>>>(s.list, s.n_list, plan.max_list, s.part, plan.n_tb, s.s2part_full,
                                                            pop_prefill_s2_gemm_splits(L), norm, N, scores, bounds, s.rank);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
+bool pop_prefill_output_supported(int d, int N, pop_dtype_t dt) { return pop_prefill_tc_supported(d, dt) && N % 8 == 0; }
+
+int pop_launch_prefill_output(void* H, int L, int d, const void* Wd, int N, const int32_t* rank, int n_active, void* Y,
+                              u32* status, int sm_count, cudaStream_t st) {
+    PrefillTcPlan plan;
+    pop_prefill_tc_plan(L, d, N, &plan);
+    mask_h_kernel<<<sm_count * 8, 256, 0, st>>>((__nv_bfloat16*)H, 2 * plan.l_pad, plan.n_pad, N, rank, n_active);
+    POP_LAUNCHED();
+    CUtensorMap mh, md;
+    int rc = make_map(&mh, H, 2 * plan.l_pad, plan.n_pad);
+    if (rc == POP_OK) rc = make_map(&md, Wd, d, N);
+    if (rc != POP_OK) return rc;
+    static thread_local int cfg_dev = -1;
+    int dev = 0;
+    POP_CUDA(cudaGetDevice(&dev));
+    if (cfg_dev != dev) {
+        POP_CUDA(cudaFuncSetAttribute(prefill_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DN_SMEM_BYTES));
+        cfg_dev = dev;
+    }
+    DownParams P;
+    P.L = L; P.d = d; P.n_tt = plan.n_tt; P.n_jt = (d + 127) / 128; P.nk = plan.n_pad / TC_BK;
+    P.lo_row = plan.l_pad;
+    P.Y = (__nv_bfloat16*)Y; P.status = status;
+    const int units = P.n_tt * P.n_jt;
+    prefill_down_kernel<<<units < sm_count ? units : sm_count, DN_THREADS, DN_SMEM_BYTES, st>>>(mh, md, P);
     POP_LAUNCHED();
     return POP_OK;
 }

@@ -65,6 +65,7 @@ SIGNATURES = {
     "pop_weights_prepare": (C.c_int, [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P, C.POINTER(_P)]),
     "pop_prefill_partition_prepared": (C.c_int, [_P, C.c_int, _P, Ratios, _P, C.POINTER(_P)]),
     "pop_weights_destroy": (C.c_int, [_P]),
+    "pop_prefill_partition_with_output": (C.c_int, [_P, C.c_int, _P, Ratios, C.c_int, _P, _P, C.POINTER(_P)]),
     "pop_partition_from_indices": (C.c_int, [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P, C.c_int, _P, C.c_int,
                                              _P, C.POINTER(_P)]),
     "pop_partition_sizes": (C.c_int, [_P] + [C.POINTER(C.c_int)] * 3),
@@ -294,6 +295,19 @@ class Weights:
         _check(lib().pop_prefill_partition_prepared(X.data_ptr(), X.shape[0], self._h, Ratios(*ratios), _stream_ptr(stream),
                                                     C.byref(out)), "pop_prefill_partition_prepared")
         return Partition(out.value, X.device)
+
+    def prefill_partition_with_output(self, X, ratios, k: int, Y=None, stream=None):
+        """pop_prefill_partition_with_output: (partition, Y [L, d]) - the partition and the prompt's own block output
+        over Retained + the k best Candidates by prefill score."""
+        torch = _torch()
+        if not (X.is_cuda and X.is_contiguous()) or _dtype_code(X) != _dtype_code(self.tensors[0]):
+            raise ValueError("X must be a contiguous CUDA tensor of the weights' dtype")
+        if Y is None:
+            Y = torch.empty_like(X)
+        out = C.c_void_p()
+        _check(lib().pop_prefill_partition_with_output(X.data_ptr(), X.shape[0], self._h, Ratios(*ratios), k, Y.data_ptr(),
+                                                       _stream_ptr(stream), C.byref(out)), "pop_prefill_partition_with_output")
+        return Partition(out.value, X.device), Y
 
     def destroy(self):
         if self._h is not None:

@@ -462,3 +462,53 @@ def test_prepared_weights_give_the_same_partition(d, N, L, dtype):
         assert np.array_equal(a.scores(), b.scores()) and np.array_equal(a.score_bounds(), b.score_bounds())
         a.destroy(); b.destroy()
     wts.destroy()
+
+
+# ------------------------------------------------------------------ the prompt's own output under the pruned structure
+@pytest.mark.parametrize("d,N,L,kfrac", [(512, 1504, 70, 0.5), (2048, 904, 40, 0.25), (320, 648, 200, 1.0), (1024, 1112, 130, 0.0)])
+def test_prefill_output_small(d, N, L, kfrac):
+    """pop_prefill_partition_with_output against the oracle's prefill_output (Sec. 3.4: Retained + the k best Candidates
+    by prefill score), several token and channel tiles with ragged tails; the partition it returns is the usual one."""
+    cfg = wl.FFNConfig("pout", d=d, N=N, dtype=wl.BF16, prompt_tokens=L, decode_steps=1, ratios=wl.Ratios(0.5, 0.2, 0.3), seed=d + L)
+    run_prefill_output_case(cfg, kfrac)
+
+
+def run_prefill_output_case(cfg, kfrac):
+    w = wl.make_ffn_workload(cfg, 1)
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    wts = pop.Weights(Wg, Wu, Wd)
+    ref = po.prefill_partition(w.X.values, *Wh, cfg.ratios.astuple())
+    k = int(round(kfrac * ref["C"].size))
+    part, Y = wts.prefill_partition_with_output(pr.to_dev(w.X), cfg.ratios.astuple(), k)
+    torch.cuda.synchronize()
+    part.check()
+    pr.check_regions(part, ref)
+    check_prefill_scores(part, ref, cfg.dtype)
+    yref = po.prefill_output(w.X.values, *Wh, ref["R"], ref["C"], ref["scores"], k)
+    err = pr.rel_err(pr.host_values(Y), yref)
+    assert err <= pr.TOL[wl.BF16], f"prompt output error {err:.3e}"
+    part.destroy()
+    wts.destroy()
+    return err
+
+
+def test_prefill_output_config2_full_size():
+    run_prefill_output_case(wl.config2(0.2), 0.5)
+
+
+def test_prefill_output_rejects_what_it_does_not_take():
+    cfg = wl.FFNConfig("pout32", d=256, N=640, dtype=wl.F32, prompt_tokens=16, decode_steps=1, seed=3)
+    w = wl.make_ffn_workload(cfg, 1)
+    wts = pop.Weights(*weights_dev(w))
+    with pytest.raises(pop.PopError) as e:
+        wts.prefill_partition_with_output(pr.to_dev(w.X), cfg.ratios.astuple(), 10)
+    assert e.value.status == pop.POP_ERR_UNSUPPORTED
+    wts.destroy()
+    cfg = wl.FFNConfig("poutk", d=256, N=640, dtype=wl.BF16, prompt_tokens=16, decode_steps=1, seed=3)
+    w = wl.make_ffn_workload(cfg, 1)
+    wts = pop.Weights(*weights_dev(w))
+    with pytest.raises(pop.PopError) as e:
+        wts.prefill_partition_with_output(pr.to_dev(w.X), cfg.ratios.astuple(), 10 ** 6)
+    assert e.value.status == pop.POP_ERR_INVALID_ARG
+    wts.destroy()
