@@ -170,3 +170,34 @@ def test_config3_full_decoder_sampled_layer_steps():
             worst = max(worst, check_layer_step(m, li, s, Wh, k))
     print(f"config 3: worst sampled layer-step output error {worst:.2e}")
     m.close()
+
+
+def test_static_decode_step_matches_the_eager_one_and_replays_as_a_graph():
+    """The graph-capturable decode step (preallocated KV cache, device-side position) against the eager one on the same
+    model and tokens, first launched eagerly, then captured once and replayed."""
+    cfg = dec.DecoderConfig(n_layers=2, d=2048, n_heads=16, N=2816, vocab=256, seed=7)
+    ratios = dec.ratios_for(0.2)
+    n_in, n_out = 24, 6
+    ids = dec.seeded_ids(cfg, n_in + n_out + 1, 4, "cuda:0")
+    m = dec.Decoder(cfg, ffn="pop", ratios=ratios)
+    m.prefill(ids[:n_in])
+    want = [m.decode(ids[n_in + s: n_in + s + 1], s)[0].float().clone() for s in range(n_out)]
+    m.reset()
+    m.prefill(ids[:n_in])
+    m.begin_static(ids, n_in + n_out + 4)
+    got = [m.step_static()[0].float().clone() for _ in range(2)]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        out = m.step_static()
+    for s in range(2, n_out):
+        graph.replay()
+        torch.cuda.synchronize()
+        got.append(out[0].float().clone())
+    for p in m.parts:
+        p.check()
+    for s in range(n_out):
+        cos = float(torch.nn.functional.cosine_similarity(got[s], want[s], dim=0))
+        assert cos > 0.9999, f"step {s}: cosine {cos}"
+    m.close()
