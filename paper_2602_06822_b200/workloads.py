@@ -200,6 +200,43 @@ def make_ffn_workload(cfg: FFNConfig, steps: Optional[int] = None) -> FFNWorkloa
                        make_prefill_input(cfg), make_decode_inputs(cfg, steps))
 
 
+def make_adversarial_case(kind: str, d: int, N: int, L: int, steps: int, batch: int = 1, seed: int = 0) -> FFNWorkload:
+    """Inputs built to strain reduced-precision accumulation (they only draw and arrange numbers):
+      "heavy_tail"        activations scaled per hidden channel by |t_3| (a few massive channels), at prefill AND at
+                          every decode step, the last step i.i.d. t_3;
+      "cancellation"      gate / up rows whose first half is about +c and second half about -c against activations
+                          near 1: partial sums of several hundred that cancel to order one;
+      "mixed_magnitudes"  activations alternating between about 1e-3 and about 1e3 along the hidden axis.
+    """
+    rng = np.random.Generator(np.random.PCG64([seed, 909]))
+    cfg = FFNConfig(f"adv_{kind}", d=d, N=N, dtype=BF16, prompt_tokens=L, decode_steps=steps, batch=batch,
+                    ratios=Ratios(0.45, 0.25, 0.30), seed=seed)
+    Wg = rng.standard_normal((N, d), dtype=np.float32) * np.float32(0.02)
+    Wu = rng.standard_normal((N, d), dtype=np.float32) * np.float32(0.02)
+    Wd = rng.standard_normal((d, N), dtype=np.float32) * np.float32(0.02)
+    X = rng.standard_normal((L * batch, d), dtype=np.float32)
+    xs = rng.standard_normal((steps, batch, d), dtype=np.float32)
+    if kind == "heavy_tail":
+        a = np.abs(rng.standard_t(3.0, size=d)).astype(np.float32)
+        X *= a[None, :]
+        xs *= a[None, None, :]
+        xs[-1] = rng.standard_t(3.0, size=(batch, d)).astype(np.float32)
+    elif kind == "cancellation":
+        sign = np.where(np.arange(d) < d // 2, 1.0, -1.0).astype(np.float32)
+        Wg = Wg + np.float32(0.5) * sign[None, :]
+        Wu = Wu + np.float32(0.25) * sign[None, :]
+        X = np.float32(1.0) + np.float32(0.01) * X
+        xs = np.float32(1.0) + np.float32(0.01) * xs
+    elif kind == "mixed_magnitudes":
+        scale = np.where(np.arange(d) % 2 == 0, 1e-3, 1e3).astype(np.float32)
+        X *= scale[None, :]
+        xs *= scale[None, None, :]
+    else:
+        raise ValueError(kind)
+    return FFNWorkload(cfg, FFNWeights(as_array(Wg, BF16), as_array(Wu, BF16), as_array(Wd, BF16)),
+                       as_array(X, BF16), as_array(xs, BF16))
+
+
 # --------------------------------------------------------------------------- MoE layer (config 4)
 @dataclass
 class MoEWorkload:

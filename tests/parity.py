@@ -4,10 +4,14 @@ Comparison rules (stated here once, used by every parity test):
   * index sets (regions, selected candidates) must be equal arrays, except that ids may swap
     across a rank boundary when their ORACLE scores lie within 1e-6 relative of the oracle's
     score at that boundary (allowance for near-ties: such scores are equal for every practical purpose);
-  * outputs: err_j = |y_j - yref_j| / max(|yref_j|, 1e-2 * max_j |yref_j|); max_j err_j must be
+  * outputs: err_j = |y_j - yref_j| / max(|yref_j|, floor * max_j |yref_j|); max_j err_j must be
     <= 1e-4 for fp32 and <= 2e-2 for bf16.  The floor keeps the measure meaningful for outputs
     that happen to lie near zero, where an fp32 accumulation has an absolute, not a relative,
-    error.
+    error.  bf16 results are gated with floor = 1e-3; fp32 results with floor = 1e-2: an fp32
+    accumulation of n products carries an absolute error of about sqrt(n) 2^-24 of the terms'
+    root-sum-square, i.e. a few 1e-6 of a typical |y_j|, which measured against 1e-3 of the
+    largest output is already of the order of the 1e-4 gate itself.  The full-size tests print the
+    worst error under both floors and the normwise error.
 """
 import numpy as np
 import torch
@@ -15,6 +19,7 @@ import torch
 from paper_2602_06822_b200 import workloads as wl
 
 TOL = {wl.F32: 1e-4, wl.BF16: 2e-2}
+FLOOR = {wl.F32: 1e-2, wl.BF16: 1e-3}
 SWAP_RTOL = 1e-6
 
 
@@ -30,14 +35,22 @@ def host_values(t: torch.Tensor) -> np.ndarray:
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-def rel_err(y: np.ndarray, yref: np.ndarray) -> float:
+def rel_err(y: np.ndarray, yref: np.ndarray, floor: float = 1e-3) -> float:
     yref = np.asarray(yref, dtype=np.float64)
     y = np.asarray(y, dtype=np.float64)
     scale = np.max(np.abs(yref))
     if scale == 0.0:
         return float(np.max(np.abs(y)))
-    den = np.maximum(np.abs(yref), 1e-2 * scale)
+    den = np.maximum(np.abs(yref), floor * scale)
     return float(np.max(np.abs(y - yref) / den))
+
+
+def bf16_ulp_distance(a: torch.Tensor, b: torch.Tensor) -> int:
+    """Largest distance, in bf16 representable values, between corresponding elements of two bf16 tensors."""
+    def ordinal(t):
+        v = t.contiguous().view(torch.int16).to(torch.int32) & 0xFFFF
+        return torch.where(v >= 0x8000, 0x8000 - v, v)          # negative values below zero, in order
+    return int((ordinal(a) - ordinal(b)).abs().max())
 
 
 def normwise_err(y, yref) -> float:

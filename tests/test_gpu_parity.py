@@ -74,12 +74,14 @@ def check_prefill_scores(part, ref, dtype):
     return int(ex.sum())
 
 
-def run_decode_parity(w, part, R, C, steps, k, Wh):
+def run_decode_parity(w, part, R, C, steps, k, Wh, floor=None):
     cfg = w.cfg
     dev = torch.device("cuda:0")
     mask = torch.empty(max(part.n_cand, 1), dtype=torch.uint8, device=dev)[:part.n_cand]
     sel = torch.empty(max(k, 1), dtype=torch.int32, device=dev)[:k]
     worst, swaps = 0.0, 0
+    worst_other, worst_norm = 0.0, 0.0
+    floor = pr.FLOOR[cfg.dtype] if floor is None else floor
     for t in range(steps):
         x = pr.to_dev(w.xs, index=t)
         mask.fill_(7)
@@ -95,9 +97,14 @@ def run_decode_parity(w, part, R, C, steps, k, Wh):
             active = np.sort(np.concatenate([R, s]))
             yref = po.masked_ffn(w.xs.values[t], *Wh, active)
         swaps += sw
-        worst = max(worst, pr.rel_err(pr.host_values(y), yref))
+        yh = pr.host_values(y)
+        worst = max(worst, pr.rel_err(yh, yref, floor))
+        worst_other = max(worst_other, pr.rel_err(yh, yref, 1e-3 if floor != 1e-3 else 1e-2))
+        worst_norm = max(worst_norm, pr.normwise_err(yh, yref))
         check_streamed_bounds(part, o, k)
     part.check()
+    print(f"[{cfg.name} d={cfg.d} N={cfg.N} B={cfg.batch} steps={steps}] worst output error: {worst:.2e} (floor {floor:g}), "
+          f"{worst_other:.2e} (floor {1e-3 if floor != 1e-3 else 1e-2:g}), normwise {worst_norm:.2e}; near-tie swaps {swaps}")
     assert worst <= pr.TOL[cfg.dtype], f"max relative output error {worst:.3e}"
     return worst, swaps
 
@@ -181,7 +188,7 @@ def test_zero_pruning_equals_dense_ffn_on_gpu():
     ref = torch.nn.functional.linear(
         torch.nn.functional.silu(torch.nn.functional.linear(x.double(), Wg.double()))
         * torch.nn.functional.linear(x.double(), Wu.double()), Wd.double())
-    assert pr.rel_err(pr.host_values(y), ref.cpu().numpy()) <= 1e-4
+    assert pr.rel_err(pr.host_values(y), ref.cpu().numpy(), pr.FLOOR[wl.F32]) <= 1e-4
     part.destroy()
 
 
@@ -210,7 +217,7 @@ def test_exact_ties_break_by_lower_channel_index(dtype, d):
             o = po.decode_step(w.xs.values[t], *Wh, ret, cand, k)
             assert np.array_equal(sel.cpu().numpy(), o["sel"])
             assert np.array_equal(mask.cpu().numpy(), o["mask"])
-            assert pr.rel_err(pr.host_values(y), o["y"]) <= pr.TOL[dtype]
+            assert pr.rel_err(pr.host_values(y), o["y"], pr.FLOOR[dtype]) <= pr.TOL[dtype]
     part.check()
     part.destroy()
 
@@ -247,7 +254,10 @@ def test_partition_from_indices_and_argument_errors():
 
 
 @pytest.mark.parametrize("d", [512, 2048])
-def test_repeated_steps_are_bit_identical_in_mask_and_close_in_output(d):
+def test_repeated_steps_are_bit_identical_in_mask_and_within_two_ulps_in_output(d):
+    """The same step twice: equal masks, and outputs that differ by at most two bf16 values (the partial sums reach the
+    fp32 accumulator in the order the SMs deliver them, so the last bit of an fp32 sum, and with it a rounding to
+    bf16, may differ; anything larger would point at a race)."""
     cfg = wl.FFNConfig("rep", d=d, N=1024, dtype=wl.BF16, prompt_tokens=32, decode_steps=1, seed=5)
     w = wl.make_ffn_workload(cfg)
     Wg, Wu, Wd = weights_dev(w)
@@ -255,20 +265,21 @@ def test_repeated_steps_are_bit_identical_in_mask_and_close_in_output(d):
     x = pr.to_dev(w.xs, index=0)
     k = part.n_cand // 2
     m1 = torch.zeros(part.n_cand, dtype=torch.uint8, device="cuda:0")
-    m2 = torch.zeros_like(m1)
     y1 = pop.decode_step(part, x, k, mask_out=m1).clone()
-    y2 = pop.decode_step(part, x, k, mask_out=m2).clone()
-    assert torch.equal(m1, m2)
-    assert pr.rel_err(pr.host_values(y2), pr.host_values(y1)) <= 1e-2
+    for rep in range(8):
+        m2 = torch.zeros_like(m1)
+        y2 = pop.decode_step(part, x, k, mask_out=m2).clone()
+        assert torch.equal(m1, m2)
+        assert pr.bf16_ulp_distance(y1, y2) <= 2
     part.destroy()
 
 
 # ------------------------------------------------------------------ full-size workloads
 @pytest.mark.parametrize("r", [0.2, 0.4])
-def test_config2_full_size(r):
+def test_config2_full_size(r, decode_impl):
     cfg = wl.config2(r)
     assert po.region_sizes(cfg.N, cfg.ratios.astuple())[:2] == ((8257, 1100) if r == 0.2 else (6056, 1100))
-    run_case(cfg, steps=6)
+    run_case(cfg, steps=32 if decode_impl == "stream" else 6)
 
 
 @pytest.mark.parametrize("batch", [1, 8])
@@ -321,7 +332,7 @@ def run_moe_case(cfg, n_experts, steps):
             parts[e].check()
             oe = [po_e for po_e in o["per_expert"] if po_e[0] == e][0][2]
             pr.check_selection(sel.cpu().numpy(), mask.cpu().numpy(), C, oe, k)
-            assert pr.rel_err(pr.host_values(ye), oe["y"]) <= pr.TOL[cfg.dtype]
+            assert pr.rel_err(pr.host_values(ye), oe["y"], pr.FLOOR[cfg.dtype]) <= pr.TOL[cfg.dtype]
             y += float(wts[j]) * ye.double()
         # The combined output: every expert output arrives rounded to bf16 (2^-9 of its own magnitude), which is
         # an absolute error for the weighted sum where the experts cancel; it is judged normwise.
@@ -337,9 +348,10 @@ def test_moe_small():
     run_moe_case(cfg, n_experts=4, steps=3)
 
 
-def test_config4_moe_full_size():
-    cfg = wl.config4_expert(0.2)
-    run_moe_case(cfg, n_experts=8, steps=2)
+@pytest.mark.parametrize("r", [0.2, 0.4])
+def test_config4_moe_full_size(r):
+    cfg = wl.config4_expert(r)
+    run_moe_case(cfg, n_experts=8, steps=4)
 
 
 @pytest.mark.gpu
@@ -512,3 +524,27 @@ def test_prefill_output_rejects_what_it_does_not_take():
         wts.prefill_partition_with_output(pr.to_dev(w.X), cfg.ratios.astuple(), 10 ** 6)
     assert e.value.status == pop.POP_ERR_INVALID_ARG
     wts.destroy()
+
+
+# ------------------------------------------------------------------ inputs built to strain the error bounds
+@pytest.mark.parametrize("batch", [1, 3])
+@pytest.mark.parametrize("kind", ["heavy_tail", "cancellation", "mixed_magnitudes"])
+def test_error_bounds_hold_on_adversarial_inputs(kind, batch):
+    """Regions and masks are decided on scores that went through the tensor cores in reduced precision, each with a bound
+    of its error; exactness rests on those bounds.  Here they meet heavy-tailed activations at decode time, rows whose
+    terms cancel from partial sums of several hundred down to order one, and activations that mix 1e-3 with 1e3.
+    Prefill scores must lie within a quarter of their bounds and the regions equal the oracle's; at every decode step
+    the masks equal the oracle's and, under the streaming kernel, |streamed - exact| stays within a quarter of the
+    streamed bound.  The outputs of these constructed cases sum terms of very different magnitude (the cancellation
+    case reaches 2.3e-2 on one near-zero output under the 1e-3 floor, 4.5e-3 under 1e-2, 2.7e-3 normwise), so they
+    are judged with the 1e-2 floor."""
+    w = wl.make_adversarial_case(kind, d=2048, N=768, L=40, steps=4, batch=batch, seed=23)
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, w.cfg.ratios.astuple())
+    ref = po.prefill_partition(w.X.values, *Wh, w.cfg.ratios.astuple())
+    check_prefill_scores(part, ref, wl.BF16)
+    pr.check_regions(part, ref)
+    R, C, _ = part.indices()
+    run_decode_parity(w, part, R, C, 4, part.n_cand // 2, Wh, floor=1e-2)
+    part.destroy()
