@@ -54,7 +54,7 @@ typedef struct pop_weights pop_weights_t;
 /*
  * Process-wide settings (host only; the paper has no counterpart: they choose among the library's kernels).
  *   decode_kernel   which decode kernel family serves partitions created from now on.  POP_DECODE_AUTO: the
- *                   streaming kernel for bf16 partitions with d in {2048, 4096, 5120} and at most 1536
+ *                   streaming kernel for bf16 partitions with d in {2048, 4096, 5120} and at most 3072
  *                   candidates, the fused persistent kernel or, where that does not fit, the multi-kernel
  *                   path for everything else; POP_DECODE_FUSED / POP_DECODE_SIMPLE force those two.
  *   launch_mode     how every later step of the streaming kernel is launched.  Its CTAs wait on one
@@ -244,7 +244,7 @@ int pop_partition_destroy(pop_partition_t* p);
  * One partition serves one stream at a time (its scratch and counters are shared by its steps).
  * Two steps of the same call sequence may differ in the last bit of y: partial sums are added to
  * the fp32 accumulator in the order the SMs deliver them; the mask does not depend on that order.
- * The default kernel for bf16 partitions with d in {2048, 4096, 5120} and at most 1536 candidates is
+ * The default kernel for bf16 partitions with d in {2048, 4096, 5120} and at most 3072 candidates is
  * launched so that its CTAs may take over SMs from the previous kernel of the stream; callers that
  * keep other streams busy on the same device should choose POP_LAUNCH_COOPERATIVE (pop_set_config):
  * a step whose CTAs cannot all be resident ends with POP_ERR_TIMEOUT at the next

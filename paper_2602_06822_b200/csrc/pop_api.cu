@@ -202,10 +202,10 @@ static int partition_alloc(int d, int N, pop_dtype_t dt, int n_ret, int n_cand, 
     const size_t row = (size_t)d * p->es;
     // pop_config_t.decode_kernel (as it stands when the partition is created) picks the decode kernel family.
     // POP_DECODE_AUTO: tiled layout + the dataflow kernel of pop_decode_stream.cu for the bf16 shapes it takes (its
-    // one-warp selection holds up to 1536 candidate keys), row layout + the fused / simple kernels for every other
+    // one-warp selection holds up to pop_stream_max_candidates() = 3072 keys), row layout + the fused / simple kernels for every other
     // shape; POP_DECODE_FUSED / POP_DECODE_SIMPLE: row layout and those kernels for all shapes.
     const int want = pop_config_snapshot().decode_kernel;
-    p->layout = (want == POP_DECODE_AUTO && pop_stream_layout_supported(d, dt) && n_cand <= 1536) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
+    p->layout = (want == POP_DECODE_AUTO && pop_stream_layout_supported(d, dt) && n_cand <= pop_stream_max_candidates()) ? POP_LAYOUT_TILED : POP_LAYOUT_ROWS;
     p->force_simple = want == POP_DECODE_SIMPLE;
     p->n_rt = (n_ret + 7) / 8;
     p->n_cg = (n_ret + 15) / 16;

@@ -206,6 +206,7 @@ int pop_launch_prefill_output(void* H, int L, int d, const void* Wd, int N, cons
                               u32* status, int sm_count, cudaStream_t st);
 // pop_decode_stream.cu (bf16 partitions in the tiled layout)
 bool pop_stream_layout_supported(int d, pop_dtype_t dt);
+int pop_stream_max_candidates();          // the streaming kernel's selection warp holds this many candidate keys
 int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void* y,
                              uint8_t* mask_out, int32_t* sel_out, cudaStream_t st);
 // pop_decode_simple.cu (multi-kernel path, any accepted shape)

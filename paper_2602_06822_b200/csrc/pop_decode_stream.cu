@@ -60,7 +60,10 @@ constexpr int SLOT = 512;                  // bytes one warp copies per cp.async
 constexpr int RING_GROUPS = 3;             // depth of a consumer warp's copy ring in phase 2 (deeper rings measured slower)
 constexpr int P2_MACRO = 4;                // largest phase-2 claim, in groups of 16 retained channels
 constexpr int P2_WINDOW = 2 * MAXG;        // groups the scheduler may stage beyond the copy ring (shallower measured slower)
-constexpr int KPL = 48;                    // candidate keys per lane of a selection warp: n_cand <= 32 * KPL
+// Candidate keys per lane of a selection warp (n_cand <= 32 * KPL): the kernel is built for two sizes, because the
+// larger one costs the common case (partition fraction 0.1: about 1100 candidates) 1.3 us per step.
+constexpr int KPL_SMALL = 48, KPL_LARGE = 96;
+constexpr int SEL_BATCH = 24;              // keys a lane fetches at once (independent loads); KPL is a multiple of it
 
 enum { T_P1_CAND = 0, T_P1_RET = 1, T_P2_RET = 2, T_P2_CAND = 3, T_END = 4 };
 enum { ERR_DESC = 11, ERR_PART_FULL = 12, ERR_FLAG = 13, ERR_SELECT_FLAG = 14, ERR_THROTTLE = 15, ERR_PART_FREE = 16,
@@ -91,7 +94,8 @@ struct StreamParams {
     int off_part, off_hfrag, off_rows, off_ystage, off_sel, off_ctrl;
 };
 
-struct Ctrl {
+template <int KPL>
+struct CtrlT {
     int4 desc[ND];
     u64 bar_full[NPB_MAX];         // the consumer warps' partial sums in buffer b are complete (NCW arrivals)
     int2 part_hdr[NPB_MAX];        // (type, unit id) of the unit in buffer b
@@ -203,6 +207,7 @@ __device__ __forceinline__ u64 h_word(float v, u32 epoch) { return (u64)__float_
 #define POP_RAISE(code) do { ctrl->abort = 1; atomicExch(gerr, (u32)(code)); } while (0)
 
 // Polls an h word until it carries the epoch of this step (bounded; ok = false on expiry or abort).
+template <typename Ctrl>
 __device__ __noinline__ u64 poll_h(const u64* p, u32 epoch, Ctrl* ctrl, u32* gerr, unsigned long long wait_ns, bool& ok) {
     PopWaitClock sp;
     for (;;) {
@@ -298,8 +303,10 @@ __device__ __noinline__ void refine_job(const StreamParams& P, int c, int e, int
 // instructions (rolled loops; lane owns candidates lane + 32 j) and fetches in batches of
 // independent loads.
 // ---------------------------------------------------------------------------------------------
-__device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, unsigned char* smem, int lane,
+template <int KPL>
+__device__ __noinline__ bool selection_main(const StreamParams& P, CtrlT<KPL>* ctrl, unsigned char* smem, int lane,
                                             int cta, int G) {
+    static_assert(KPL % SEL_BATCH == 0, "the key fetch loop runs in whole batches");
     const int n = P.n_cand, k = P.k;
     const int rows = (n + 31) >> 5;
     u32* gerr = P.sync + SYNC_ERROR;
@@ -336,15 +343,15 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, u
         float mm = 0.f;
         u32 kor = 0u, kand = ~0u;
 #pragma unroll 1
-        for (int j0 = 0; j0 < rows; j0 += KPL / 2) {
-            uint2 kv[KPL / 2];
+        for (int j0 = 0; j0 < rows; j0 += SEL_BATCH) {
+            uint2 kv[SEL_BATCH];
 #pragma unroll
-            for (int t = 0; t < KPL / 2; ++t) {
+            for (int t = 0; t < SEL_BATCH; ++t) {
                 const int i = lane + 32 * (j0 + t);
                 kv[t] = i < n ? __ldcg(P.km + i) : make_uint2(0u, 0u);
             }
 #pragma unroll
-            for (int t = 0; t < KPL / 2; ++t) {
+            for (int t = 0; t < SEL_BATCH; ++t) {
                 kr[32 * (j0 + t)] = kv[t].x;
                 if (lane + 32 * (j0 + t) < n) { kor |= kv[t].x; kand &= kv[t].x; }
                 mm = fmaxf(mm, __uint_as_float(kv[t].y));
@@ -526,8 +533,9 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, Ctrl* ctrl, u
 // The kernel.  GS = d / 1024 = 512-byte slots per warp and copy group; NBLK = n-blocks of 8
 // columns used in phase 2 (batch <= 4 * NBLK).
 // ---------------------------------------------------------------------------------------------
-template <int GS, int NBLK>
+template <int GS, int NBLK, int KPL>
 __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const StreamParams P) {
+    using Ctrl = CtrlT<KPL>;
     constexpr int GSL = GS * (16 / NCW);   // 512-byte slots per warp and copy group
     constexpr int S = 4 * GSL;             // slots per warp in a phase-1 unit
     constexpr int CPR = 2 * GSL;            // 16-byte chunks per candidate row and warp in phase 2
@@ -914,7 +922,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         POP_TRACE(14);
     } else if (warp == W_SEL) {
         // ================================================================= selection warp
-        selection_main(P, ctrl, smem, lane, cta, G);
+        selection_main<KPL>(P, ctrl, smem, lane, cta, G);
     } else {
         // ================================================================= consumer warps
         const int w = warp;
@@ -1282,9 +1290,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
 
 inline int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
-template <int GS, int NBLK>
+template <int GS, int NBLK, int KPL>
 int launch_stream(StreamParams& P, const pop_partition* p, cudaStream_t st) {
-    auto kern = pop_decode_stream_kernel<GS, NBLK>;
+    using Ctrl = CtrlT<KPL>;
+    auto kern = pop_decode_stream_kernel<GS, NBLK, KPL>;
     // shared-memory layout: [ring][part][hfrag][rows][ystage][ctrl]
     const int GSL = GS * (16 / NCW);
     const int NPB = NBLK == 1 ? 3 : 2;
@@ -1362,6 +1371,8 @@ extern "C" int pop_debug_stream_trace(unsigned long long* h_out, int ctas) {
 }
 #endif
 
+int pop_stream_max_candidates() { return 32 * KPL_LARGE; }
+
 bool pop_stream_layout_supported(int d, pop_dtype_t dt) {
     if (dt != POP_BF16 || d % 1024 != 0) return false;
     const int gs = d / 1024;
@@ -1402,7 +1413,7 @@ int pop_launch_decode_stream(pop_partition* p, const void* x, int B, int k, void
     P.wait_ns = 1000ull * (unsigned long long)pop_config_snapshot().wait_budget_us;
     const int gs = p->d / 1024;
     const int nblk = B <= 4 ? 1 : 2;
-#define POP_CASE(G_, N_) if (gs == G_ && nblk == N_) return launch_stream<G_, N_>(P, p, st);
+#define POP_CASE(G_, N_) if (gs == G_ && nblk == N_) return p->n_cand <= 32 * KPL_SMALL ? launch_stream<G_, N_, KPL_SMALL>(P, p, st) : launch_stream<G_, N_, KPL_LARGE>(P, p, st);
     POP_CASE(2, 1) POP_CASE(2, 2) POP_CASE(4, 1) POP_CASE(4, 2) POP_CASE(5, 1) POP_CASE(5, 2)
 #undef POP_CASE
     return POP_ERR_UNSUPPORTED;

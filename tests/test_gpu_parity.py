@@ -548,3 +548,30 @@ def test_error_bounds_hold_on_adversarial_inputs(kind, batch):
     R, C, _ = part.indices()
     run_decode_parity(w, part, R, C, 4, part.n_cand // 2, Wh, floor=1e-2)
     part.destroy()
+
+
+# ------------------------------------------------------------------ wide candidate regions (partition fraction 0.2 and more)
+@pytest.mark.parametrize("B", [1, 4])
+def test_many_candidates_on_the_streaming_kernel(B, decode_impl):
+    """More than 1536 and up to 3072 candidates: still the streaming kernel (its selection warp holds 96 keys per lane)."""
+    cfg = wl.FFNConfig("wideC", d=2048, N=4000, dtype=wl.BF16, prompt_tokens=24, decode_steps=3, batch=B,
+                       ratios=wl.Ratios(0.25, 0.65, 0.10), seed=77)
+    assert po.region_sizes(cfg.N, cfg.ratios.astuple())[1] == 2600
+    run_case(cfg)
+
+
+def test_config2_gamma02_full_size(decode_impl):
+    """Sec. 5 "Partition Fraction": gamma = 0.2 at Llama-2-7B shapes is 2201 candidates."""
+    cfg = wl.scaled(wl.config2(0.2), ratios=wl.ratios_for(0.2, 0.2), name="cfg2_llama7b_r20_gamma20")
+    assert po.region_sizes(cfg.N, cfg.ratios.astuple())[:2] == (7707, 2201)
+    w = wl.make_ffn_workload(cfg, 4)
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    part = pop.prefill_partition(pr.to_dev(w.X), Wg, Wu, Wd, cfg.ratios.astuple())
+    if decode_impl == "stream":
+        part.streamed_scores()          # raises unless the streaming kernel serves this partition
+    ref = po.prefill_partition(w.X.values, *Wh, cfg.ratios.astuple())
+    pr.check_regions(part, ref)
+    R, C, _ = part.indices()
+    run_decode_parity(w, part, R, C, 4, part.n_cand // 2, Wh)
+    part.destroy()
