@@ -487,20 +487,44 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, CtrlT<KPL>* c
                 uex[e] = score_key(P.norm_cand[c] * sqrt(energy));
             }
             __syncwarp();
-            // rank inside the uncertain set (ulist ascends, so position order is channel order)
+            // the best ku of the uncertain set by (exact score descending, channel id ascending); ulist ascends, so
+            // position order is channel order
             const int ku = k - nin;
+            if (nu <= 64) {
+                // a few candidates: every lane ranks its own against all
 #pragma unroll 1
-            for (int e = lane; e < nu; e += 32) {
-                const u64 ke = uex[e];
-                int r = 0;
+                for (int e = lane; e < nu; e += 32) {
+                    const u64 ke = uex[e];
+                    int r = 0;
 #pragma unroll 1
-                for (int f = 0; f < nu; ++f) {
-                    const u64 kf = uex[f];
-                    r += (kf > ke || (kf == ke && f < e)) ? 1 : 0;
+                    for (int f = 0; f < nu; ++f) {
+                        const u64 kf = uex[f];
+                        r += (kf > ke || (kf == ke && f < e)) ? 1 : 0;
+                    }
+                    if (r < ku) {
+                        const int ce = ulist[e];
+                        atomicOr(&rowmask[ce >> 5], 1u << (ce & 31));
+                    }
                 }
-                if (r < ku) {
-                    const int ce = ulist[e];
-                    atomicOr(&rowmask[ce >> 5], 1u << (ce & 31));
+            } else if (ku > 0) {
+                // many (scores that the bounds cannot tell apart, e.g. all equal): a radix select on the exact keys
+                // instead of nu^2 / 32 comparisons per lane, then one ordered walk for the ties at the threshold
+                u64 thr = 0;
+                int need_eq = 0;
+                radix_select_kth<32>(uex, nu, ku < nu ? ku : nu, hist, lane, 1, thr, need_eq);
+                int eq_seen = 0;
+#pragma unroll 1
+                for (int e0 = 0; e0 < nu; e0 += 32) {
+                    const int e = e0 + lane;
+                    const bool valid = e < nu;
+                    const u64 ke = valid ? uex[e] : 0ull;
+                    const bool is_eq = valid && ke == thr;
+                    const u32 beq = __ballot_sync(0xffffffffu, is_eq);
+                    if (valid && (ke > thr || (is_eq && eq_seen + __popc(beq & lt) < need_eq))) {
+                        const int ce = ulist[e];
+                        atomicOr(&rowmask[ce >> 5], 1u << (ce & 31));
+                    }
+                    eq_seen += __popc(beq);
                 }
             }
             __syncwarp();
