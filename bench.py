@@ -199,8 +199,8 @@ def run_reference(args):
 # profiles.  The figure belongs to one version of the kernel's source: it is reported only while the source file
 # still hashes to what it was when the counters were taken, and is null otherwise.
 NCU_TRAFFIC = {
-    "llama2_7b_ffn_r20_b1": {"bytes": 235.6e6, "kernel_source": "paper_2602_06822_b200/csrc/pop_decode_stream.cu",
-                             "sha256_16": "", "summary": "profiles/pop_decode_stream_kernel_llama2_7b_r20_b1.md"},
+    "llama2_7b_ffn_r20_b1": {"bytes": 236.1e6, "kernel_source": "paper_2602_06822_b200/csrc/pop_decode_stream.cu",
+                             "sha256_16": "22c00c1a690b7b6e", "summary": "profiles/pop_decode_stream_kernel_llama2_7b_r20_b1.md"},
 }
 
 
@@ -326,7 +326,8 @@ def run_pop(args):
     pop.lib()
     # every step builds and destroys one partition per layer: let the library keep all of their memory for the next
     # step (the default keeps 1 GiB), as a serving loop with this many live layers would
-    pop.set_config(slab_cache_bytes=16 << 30)
+    pop.set_config(slab_cache_bytes=16 << 30,
+                   decode_kernel={"auto": pop.POP_DECODE_AUTO, "fused": pop.POP_DECODE_FUSED, "simple": pop.POP_DECODE_SIMPLE}[args.decode_kernel])
 
     name = args.workload
     d, N, dts, L, B, r = WORKLOADS[name]
@@ -525,7 +526,7 @@ def run_pop(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dts, "data": "synthetic",
             "config": {"workload": name, "d": d, "N": N, "batch": B, "prompt_tokens": L * B, "ratios": list(ratios),
                        "n_ret": n_ret, "n_cand": n_cand, "k": k, "layers": layers, "tokens": tokens,
-                       "slab_cache_bytes": 16 << 30,
+                       "slab_cache_bytes": 16 << 30, "decode_kernel": args.decode_kernel,
                        "l2": f"inputs larger than L2: {layers} layers x {abytes / 1e6:.1f} MB of distinct weights per token",
                        "replicas": world},
             "us_per_layer_step": us_per_ls,
@@ -589,6 +590,8 @@ def main(argv=None):
     ap.add_argument("--workload", default="llama2_7b_ffn_r20_b1", choices=sorted(WORKLOADS))
     ap.add_argument("--layers", type=int, default=8)
     ap.add_argument("--tokens", type=int, default=128)
+    ap.add_argument("--decode-kernel", default="auto", choices=["auto", "fused", "simple"],
+                    help="decode kernel family (pop_set_config): auto = the streaming kernel where it applies")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the method's variants and the gamma sweep")
     ap.add_argument("--no-workloads", action="store_true", help="skip the per_workload list")
