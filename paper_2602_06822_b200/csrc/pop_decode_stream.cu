@@ -585,8 +585,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
     }
     if (tid < NCW) { ctrl->cons_m[tid] = 0; ctrl->cons_g[tid] = 0; }
     // When launched with programmatic stream serialization the CTA may have started while the previous kernel of
-    // the stream was still running: nothing of global memory is touched before that kernel is complete.  The next
-    // kernel may be placed from now on (it takes an SM only once a CTA of this one has left it).
+    // the stream was still running: nothing that a kernel of the stream may have written is touched before that kernel
+    // is complete.  The repacked weights are the exception: they are written once, by the kernels that build the
+    // partition, which do not release their dependents early (so this kernel cannot have started before they
+    // completed), and never again; the consumer warps therefore issue the loads of their first phase-1 unit before the
+    // wait, which takes the first trip to HBM out of the step.  The next kernel may be placed from the wait on (it takes
+    // an SM only once a CTA of this one has left it).
+    constexpr int PRE_GSL = GS * (16 / NCW), PRE_S = 4 * PRE_GSL, PRE_BS = PRE_S % 16 == 0 ? 8 : 5;
+    uint4 preA[PRE_BS], preB[PRE_BS];
+    if (warp < NCW && cta < P.U1) {
+        const int tile0 = cta < P.Uc ? P.n_rt + cta : cta - P.Uc;      // this CTA's first unit (candidate tiles follow the retained ones)
+        const unsigned char* s0 = P.GUt + ((size_t)tile0 * (size_t)(P.d >> 4) + (size_t)(warp * PRE_S)) * SLOT + lane * 16;
+#pragma unroll
+        for (int j = 0; j < PRE_BS; ++j) preA[j] = ldg_stream(s0 + j * SLOT);
+#pragma unroll
+        for (int j = 0; j < PRE_BS; ++j) preB[j] = ldg_stream(s0 + (PRE_BS + j) * SLOT);
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 #ifdef POP_STREAM_TRACE
@@ -1107,14 +1121,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                 const int tile = p < P.Uc ? P.n_rt + p : p - P.Uc;        // candidate tiles follow the retained ones
                 return P.GUt + ((size_t)tile * KT + (size_t)(w * S)) * SLOT + lane * 16;
             };
+            static_assert(BS == PRE_BS, "the loads issued before the dependency wait are the first two batches");
             uint4 bufA[BS], bufB[BS];
-            if (p1_count > 0) {
-                const unsigned char* s0 = src_of(0);
 #pragma unroll
-                for (int j = 0; j < BS; ++j) bufA[j] = ldg_stream(s0 + j * SLOT);
-#pragma unroll
-                for (int j = 0; j < BS; ++j) bufB[j] = ldg_stream(s0 + (BS + j) * SLOT);
-            }
+            for (int j = 0; j < BS; ++j) { bufA[j] = preA[j]; bufB[j] = preB[j]; }      // issued at the top of the kernel
 #pragma unroll 1
             for (int i = 0; i < p1_count && ok; ++i) {
                 if (w == 0 && lane == 0) ctrl->p1_started = i + 1;
