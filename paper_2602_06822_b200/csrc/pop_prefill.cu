@@ -672,6 +672,134 @@ __global__ void __launch_bounds__(256) repack_wdtt_kernel(const __nv_bfloat16* _
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Both W_d outputs of the tiled layout in one pass over W_d: the retained fragments WdTt and the plain candidate rows
+// WdTc.  Block (sg, jc) stages W_d[64 jc .. + 63][c_lo .. c_hi) in shared memory with coalesced 16-byte loads, where
+// [c_lo, c_hi) is the span of channel ids from the first retained slot of slot group sg (128 retained slots) up to the
+// first slot of the next group (the spans tile [0, N), so every candidate lies in exactly one of them), and builds
+// from it the 8 x 4 fragment tiles of its slots and the 64-row pieces of the candidates inside the span.  W_d is read
+// once (the pruned columns inside a span ride along); the former per-element column gathers from global memory cost
+// twice the time.  A span too wide for the staging buffer (very sparse retained regions) is read from global memory
+// directly, element by element, by the same code.
+// ---------------------------------------------------------------------------------------------
+#define RWD_ROWS 64
+#define RWD_SLOTS 128
+#define RWD_SPAN_MAX 512
+
+// rows of the staged tile start 16 bytes aligned and an odd number of 16-byte units apart (8 rows fall on 8 bank groups)
+__host__ __device__ __forceinline__ int rwd_pitch_vec(int nvec) { return (nvec + 1) | 1; }
+
+template <bool STAGED>
+__device__ __forceinline__ void rwd_emit(const unsigned short* __restrict__ W, const unsigned short* tile, int pitch,
+                                         int c_lo8, int j0, int d, int N, int n_cg, int sg, const int* slot_ch,
+                                         int ca, int cb, const int32_t* __restrict__ idx_cand, uint4* __restrict__ WdTt,
+                                         __nv_bfloat16* __restrict__ WdTc) {
+    const int tid = threadIdx.x, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    // element (row jl of the block, channel offset off) of W_d
+    auto rd = [&](int jl, int off) -> u32 {
+        return STAGED ? (u32)tile[jl * pitch + off] : (u32)W[(size_t)(j0 + jl) * N + c_lo8 + off];
+    };
+    // retained fragments: warp = column group (16 slots), 4 m-tiles of 16 rows each, one 16-byte vector per lane and tile
+    const int cg8 = tid >> 5, cg = 8 * sg + cg8;
+    if (cg < n_cg) {
+        int off[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const int ch = slot_ch[16 * cg8 + 2 * t + (h & 1) + ((h >> 1) ? 8 : 0)];
+            off[h] = ch < 0 ? -1 : ch - c_lo8;
+        }
+        const int MT = d >> 6, quarter_rows = d >> 2;
+        const int q = j0 / quarter_rows, mt0 = (j0 - q * quarter_rows) >> 4;
+        uint4* out = WdTt + (((size_t)q * n_cg + cg) * MT + mt0) * 32 + lane;
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt) {
+            u32 r[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int jl = 16 * mt + g + ((e & 1) ? 8 : 0);
+                const int oa = off[2 * (e >> 1)], ob = off[2 * (e >> 1) + 1];
+                const u32 lo = oa >= 0 ? rd(jl, oa) : 0u, hi = ob >= 0 ? rd(jl, ob) : 0u;
+                r[e] = lo | (hi << 16);
+            }
+            out[mt * 32] = make_uint4(r[0], r[1], r[2], r[3]);
+        }
+    }
+    // candidate rows inside the span: 8 pieces of 8 rows each
+    for (int w = tid; w < (cb - ca) * 8; w += 256) {
+        const int c = ca + (w >> 3), rv = w & 7;
+        const int off = __ldg(idx_cand + c) - c_lo8;
+        u32 o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[e] = rd(8 * rv + 2 * e, off) | (rd(8 * rv + 2 * e + 1, off) << 16);
+        *reinterpret_cast<uint4*>(WdTc + (size_t)c * d + j0 + 8 * rv) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
+__global__ void __launch_bounds__(256) repack_wd_tiled_kernel(const __nv_bfloat16* __restrict__ Wd, int d, int N, int n_ret,
+                                                              int n_cg, int n_cand, const int32_t* __restrict__ idx_ret,
+                                                              const int32_t* __restrict__ idx_cand, uint4* __restrict__ WdTt,
+                                                              __nv_bfloat16* __restrict__ WdTc) {
+    extern __shared__ __align__(16) unsigned short rwd_tile[];     // [RWD_ROWS][pitch]
+    __shared__ int slot_ch[RWD_SLOTS];
+    __shared__ int span[2];                                        // first and last + 1 candidate of the span
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, sg = blockIdx.x, j0 = blockIdx.y * RWD_ROWS;
+    const int n_sg = gridDim.x;
+    const unsigned short* W = reinterpret_cast<const unsigned short*>(Wd);
+    if (tid < RWD_SLOTS) {
+        const int s = RWD_SLOTS * sg + tid;
+        slot_ch[tid] = s < n_ret ? idx_ret[s] : -1;
+    }
+    if (tid < 2) span[tid] = 0;
+    const int c_lo = sg == 0 ? 0 : __ldg(idx_ret + RWD_SLOTS * sg);
+    const int c_hi = sg == n_sg - 1 ? N : __ldg(idx_ret + RWD_SLOTS * (sg + 1));
+    const int c_lo8 = c_lo & ~7;
+    const int nvec = (c_hi - c_lo8 + 7) >> 3;                       // 16-byte vectors per staged row (N is a multiple of 8)
+    const bool staged = nvec * 8 <= RWD_SPAN_MAX + 8;
+    const int pitch = 8 * rwd_pitch_vec(nvec);
+    __syncthreads();
+    if (staged) {
+        // a warp per row, lanes along the row: every load of a warp is one contiguous run
+        const uint4* src = reinterpret_cast<const uint4*>(W + (size_t)(j0 + warp) * N + c_lo8) + lane;
+        uint4* dst = reinterpret_cast<uint4*>(rwd_tile + warp * pitch) + lane;
+        const size_t src_step = (size_t)N;                          // 8 rows, in 16-byte units
+        const int dst_step = pitch;
+        if (nvec <= 32) {
+            uint4 x[RWD_ROWS / 8];
+            if (lane < nvec) {
+#pragma unroll
+                for (int i = 0; i < RWD_ROWS / 8; ++i) x[i] = __ldg(src + i * src_step);
+#pragma unroll
+                for (int i = 0; i < RWD_ROWS / 8; ++i) dst[i * dst_step] = x[i];
+            }
+        } else {
+            for (int cv = lane; cv < nvec; cv += 32) {
+                uint4 x[RWD_ROWS / 8];
+#pragma unroll
+                for (int i = 0; i < RWD_ROWS / 8; ++i) x[i] = __ldg(src + i * src_step + (cv - lane));
+#pragma unroll
+                for (int i = 0; i < RWD_ROWS / 8; ++i) dst[i * dst_step + (cv - lane)] = x[i];
+            }
+        }
+    }
+    {   // candidates below the span and below its end, counted by all threads (independent loads, one latency)
+        int below_lo = 0, below_hi = 0;
+        for (int i = tid; i < n_cand; i += 256) {
+            const int v = __ldg(idx_cand + i);
+            below_lo += v < c_lo; below_hi += v < c_hi;
+        }
+        below_lo = __reduce_add_sync(0xffffffffu, below_lo); below_hi = __reduce_add_sync(0xffffffffu, below_hi);
+        if (lane == 0) { atomicAdd(&span[0], below_lo); atomicAdd(&span[1], below_hi); }
+    }
+    __syncthreads();
+    const int ca = span[0], cb = span[1];
+    if (staged) rwd_emit<true>(W, rwd_tile, pitch, c_lo8, j0, d, N, n_cg, sg, slot_ch, ca, cb, idx_cand, WdTt, WdTc);
+    else rwd_emit<false>(W, rwd_tile, pitch, c_lo8, j0, d, N, n_cg, sg, slot_ch, ca, cb, idx_cand, WdTt, WdTc);
+}
+
+static bool repack_wd_tiled_applies(const pop_partition* p) {
+    return p->n_ret > 0 && p->N % 8 == 0 && p->d % (4 * RWD_ROWS) == 0;
+}
+
 int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* Wu, const void* Wd,
                             const double* norm, cudaStream_t st) {
     const size_t row = (size_t)p->d * 2;
@@ -686,7 +814,21 @@ int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* 
                                                   p->n_cand, p->n_ct, p->idx_ret, p->idx_cand, (uint4*)GUt);
         POP_LAUNCHED();
     }
-    if (p->n_rt > 0) {
+    const bool merged = repack_wd_tiled_applies(p);
+    if (merged) {
+        const size_t smem = sizeof(unsigned short) * RWD_ROWS * 8 * rwd_pitch_vec(RWD_SPAN_MAX / 8 + 1);
+        static thread_local int cfg_dev = -1;
+        int dev = 0;
+        POP_CUDA(cudaGetDevice(&dev));
+        if (cfg_dev != dev) {
+            POP_CUDA(cudaFuncSetAttribute(repack_wd_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            cfg_dev = dev;
+        }
+        dim3 grd((p->n_ret + RWD_SLOTS - 1) / RWD_SLOTS, p->d / RWD_ROWS);
+        repack_wd_tiled_kernel<<<grd, 256, smem, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_ret, p->n_cg, p->n_cand,
+                                                       p->idx_ret, p->idx_cand, (uint4*)WdTt, (__nv_bfloat16*)WdTc);
+        POP_LAUNCHED();
+    } else if (p->n_rt > 0) {
         const size_t total2 = (size_t)4 * p->n_cg * (p->d / 64) * 32;
         const int blocks2 = (int)((total2 + 255) / 256 < 148 * 64 ? (total2 + 255) / 256 : 148 * 64);
         repack_wdtt_kernel<<<blocks2, 256, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_ret, p->n_cg,
@@ -698,10 +840,12 @@ int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* 
         repack_gu_kernel<<<p->n_cand, 256, 0, st>>>((const uint4*)Wg, (const uint4*)Wu, row_vecs, 0, p->n_cand, p->idx_cand,
                                                     p->idx_cand, (uint4*)GUc, norm, p->norm_cand, p->wnorm_cand);
         POP_LAUNCHED();
-        dim3 blk(32, 32), grd((p->n_cand + 31) / 32, (p->d + 31) / 32);
-        repack_wdt_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_cand, 0,
-                                                               p->idx_cand, p->idx_cand, (__nv_bfloat16*)WdTc);
-        POP_LAUNCHED();
+        if (!merged) {
+            dim3 blk(32, 32), grd((p->n_cand + 31) / 32, (p->d + 31) / 32);
+            repack_wdt_kernel<__nv_bfloat16><<<grd, blk, 0, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_cand, 0,
+                                                                   p->idx_cand, p->idx_cand, (__nv_bfloat16*)WdTc);
+            POP_LAUNCHED();
+        }
     }
     return POP_OK;
 }

@@ -153,10 +153,23 @@ def test_config1_full():
     (2048, 333, 9, 8, wl.BF16),
     (4096, 1500, 16, 1, wl.BF16),
     (5120, 900, 16, 2, wl.BF16),
+    # N a multiple of 8: W_d is repacked by the kernel that stages channel spans in shared memory
+    (2048, 1208, 20, 3, wl.BF16),
+    (4096, 1504, 16, 1, wl.BF16),
+    (1024, 2056, 30, 2, wl.BF16),
 ])
 def test_small_shapes(d, N, L, B, dtype):
     cfg = wl.FFNConfig(f"s{d}x{N}", d=d, N=N, dtype=dtype, prompt_tokens=L, decode_steps=5, batch=B,
                        ratios=wl.Ratios(0.45, 0.25, 0.30), seed=d + N)
+    run_case(cfg)
+
+
+@pytest.mark.parametrize("ratios", [(0.05, 0.25, 0.70), (0.02, 0.08, 0.90), (0.90, 0.05, 0.05)])
+def test_sparse_and_dense_retained_regions_tiled(ratios):
+    """Few retained channels: the channel span of one group of retained slots is wider than the repacking kernel's
+    staging buffer and it reads W_d directly; many: narrow spans."""
+    cfg = wl.FFNConfig("span", d=2048, N=4096, dtype=wl.BF16, prompt_tokens=20, decode_steps=3, batch=2,
+                       ratios=wl.Ratios(*ratios), seed=29)
     run_case(cfg)
 
 
