@@ -69,8 +69,11 @@ typedef struct pop_weights pop_weights_t;
  *                   pop_partition_check as POP_ERR_TIMEOUT; it never hangs.
  *   slab_cache_bytes  device memory of destroyed partitions that the library keeps for the next partition
  *                   of the same size (default 1 GiB; 0 = keep nothing, and releases what is held).
- * pop_release_cached_memory() gives all of that memory back to the driver at once (it calls cudaFree,
- * which synchronises the device).
+ * The temporaries of a prefill come from a stream-ordered memory pool of the library's own (one per device)
+ * that keeps what it has allocated while the device is idle: a few MB, tens of MB after
+ * pop_prefill_partition_with_output.
+ * pop_release_cached_memory() gives all of that memory (cached slabs and the pool's unused memory) back to
+ * the driver at once (it calls cudaFree, which synchronises the device).
  */
 typedef enum { POP_DECODE_AUTO = 0, POP_DECODE_FUSED = 1, POP_DECODE_SIMPLE = 2 } pop_decode_kernel_t;
 typedef enum { POP_LAUNCH_PDL = 0, POP_LAUNCH_COOPERATIVE = 1, POP_LAUNCH_PLAIN = 2 } pop_launch_mode_t;

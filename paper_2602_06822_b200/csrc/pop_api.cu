@@ -71,6 +71,52 @@ const DeviceInfo& device_info(int device) {
 }
 }  // namespace
 
+// Temporaries of the prefill come from a stream-ordered pool of the library's own, one per device, that keeps its
+// memory when the device goes idle: the device's default pool hands everything back to the driver at each
+// synchronisation (release threshold 0), and the first allocation after one then costs several hundred microseconds
+// of host time during which the GPU has nothing to do.  What the pool holds is the largest set of temporaries in
+// flight (a few MB; tens of MB with pop_prefill_partition_with_output); pop_release_cached_memory() trims it.  If the
+// pool cannot be created the default pool serves.
+namespace {
+struct TempPool { int tried; cudaMemPool_t pool; };
+TempPool g_temp_pools[64];
+std::mutex g_temp_pool_mutex;
+
+cudaMemPool_t temp_pool(int device) {
+    if (device < 0 || device >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_temp_pool_mutex);
+    TempPool& t = g_temp_pools[device];
+    if (!t.tried) {
+        t.tried = 1;
+        cudaMemPoolProps props;
+        memset(&props, 0, sizeof(props));
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = device;
+        cudaMemPool_t pool = nullptr;
+        if (cudaMemPoolCreate(&pool, &props) == cudaSuccess) {
+            unsigned long long keep = ~0ull;
+            if (cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep) == cudaSuccess) t.pool = pool;
+            else cudaMemPoolDestroy(pool);
+        }
+        (void)cudaGetLastError();
+    }
+    return t.pool;
+}
+
+cudaError_t temp_alloc(void** ptr, size_t bytes, int device, cudaStream_t st) {
+    cudaMemPool_t pool = temp_pool(device);
+    return pool ? cudaMallocFromPoolAsync(ptr, bytes, pool, st) : cudaMallocAsync(ptr, bytes, st);
+}
+
+void temp_pools_trim() {
+    std::lock_guard<std::mutex> lock(g_temp_pool_mutex);
+    for (int i = 0; i < 64; ++i)
+        if (g_temp_pools[i].pool) cudaMemPoolTrimTo(g_temp_pools[i].pool, 0);
+}
+}  // namespace
+
 static bool aligned16(const void* p) { return (((uintptr_t)p) & 15u) == 0; }
 
 static int check_shape(int d, int N, pop_dtype_t dt) {
@@ -171,6 +217,7 @@ extern "C" int pop_set_config(const pop_config_t* in) {
 
 extern "C" int pop_release_cached_memory(void) {
     slab_flush();
+    temp_pools_trim();
     return POP_OK;
 }
 
@@ -356,7 +403,7 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
         t_part = tmp.take(sizeof(double) * (size_t)tp.max_list * tp.n_tb);
     }
     unsigned char* tb = nullptr;
-    cudaError_t e = cudaMallocAsync((void**)&tb, tmp.total, st);
+    cudaError_t e = temp_alloc((void**)&tb, tmp.total, p->device, st);
     if (e != cudaSuccess) {
         pop_set_cuda_error(e, "cudaMallocAsync");
         partition_free_now(p, st);
@@ -489,7 +536,7 @@ extern "C" int pop_partition_from_indices(const void* Wg, const void* Wu, const 
     free(h_pruned);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "index upload"); partition_free_now(p, st); return POP_ERR_CUDA; }
     double* norm = nullptr;
-    e = cudaMallocAsync((void**)&norm, sizeof(double) * (size_t)N, st);
+    e = temp_alloc((void**)&norm, sizeof(double) * (size_t)N, p->device, st);
     if (e != cudaSuccess) { pop_set_cuda_error(e, "cudaMallocAsync"); partition_free_now(p, st); return POP_ERR_ALLOC; }
     rc = pop_launch_colnorm(Wd, d, N, dtype, norm, st);
     if (rc == POP_OK) rc = p->layout == POP_LAYOUT_TILED ? pop_launch_repack_tiled(p, Wg, Wu, Wd, norm, st)
