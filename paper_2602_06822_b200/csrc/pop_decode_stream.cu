@@ -813,33 +813,46 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                 __syncwarp();
                 // their h as mma B fragments (written by the reducers of the candidate units, all of which the
                 // selection has waited for; the epoch tag is checked all the same)
-                for (int gi = 0; gi < ng && ok; ++gi) {
+                // All words of the unit are fetched at once (one memory round trip), then any word whose tag is old
+                // is polled.  A mask word selects at most 32 rows: two groups.
+                u64 hw[2][NBLK][4];
 #pragma unroll
-                    for (int nb = 0; nb < NBLK; ++nb) {
-                        const int n = g8 + 8 * nb, bb = n >> 1, part = n & 1;
-                        float v[4];
+                for (int gi = 0; gi < 2; ++gi)
+#pragma unroll
+                    for (int nb = 0; nb < NBLK; ++nb)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const int kk = 2 * t4 + (e & 1) + (e >> 1) * 8;
-                            const int sc = rw[16 * gi + kk];
-                            v[e] = 0.f;
-                            if (sc >= 0 && bb < B) {
-                                const u64* hp = P.h + (size_t)bb * P.h_stride + P.n_ret_pad + sc;
-                                PopWaitClock sp;
-                                for (;;) {
-                                    const u64 hw = __ldcg(hp);
-                                    if ((u32)(hw >> 32) == epoch) { v[e] = __uint_as_float((u32)hw); break; }
-                                    if (ctrl->abort) { ok = false; break; }
-                                    if (sp.expired(P.wait_ns)) { POP_RAISE(ERR_FLAG); ok = false; break; }
-                                    __nanosleep(64);
-                                }
+                            const int bb = (g8 + 8 * nb) >> 1;
+                            const int sc = gi < ng ? rw[16 * gi + 2 * t4 + (e & 1) + (e >> 1) * 8] : -1;
+                            hw[gi][nb][e] = (sc >= 0 && bb < B) ? __ldcg(P.h + (size_t)bb * P.h_stride + P.n_ret_pad + sc)
+                                                                : ((u64)epoch << 32);       // value 0
+                        }
+#pragma unroll
+                for (int gi = 0; gi < 2; ++gi)
+#pragma unroll
+                    for (int nb = 0; nb < NBLK; ++nb)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if ((u32)(hw[gi][nb][e] >> 32) != epoch) {
+                                const int bb = (g8 + 8 * nb) >> 1;
+                                const int sc = rw[16 * gi + 2 * t4 + (e & 1) + (e >> 1) * 8];
+                                hw[gi][nb][e] = poll_h(P.h + (size_t)bb * P.h_stride + P.n_ret_pad + sc, epoch, ctrl, gerr, P.wait_ns, ok);
                             }
                         }
-                        hfrag[((dslot * MAXG + gi) * NBLK + nb) * 32 + lane] =
-                            make_uint2(pack2(split_bits(v[0], part), split_bits(v[1], part)),
-                                       pack2(split_bits(v[2], part), split_bits(v[3], part)));
+#pragma unroll
+                for (int gi = 0; gi < 2; ++gi)
+#pragma unroll
+                    for (int nb = 0; nb < NBLK; ++nb) {
+                        if (gi < ng) {
+                            const int part = (g8 + 8 * nb) & 1;
+                            float v[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) v[e] = __uint_as_float((u32)hw[gi][nb][e]);
+                            hfrag[((dslot * MAXG + gi) * NBLK + nb) * 32 + lane] =
+                                make_uint2(pack2(split_bits(v[0], part), split_bits(v[1], part)),
+                                           pack2(split_bits(v[2], part), split_bits(v[3], part)));
+                        }
                     }
-                }
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
             }
