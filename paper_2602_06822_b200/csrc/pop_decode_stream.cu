@@ -600,6 +600,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         for (int j = 0; j < PRE_BS; ++j) preA[j] = ldg_stream(s0 + j * SLOT);
 #pragma unroll
         for (int j = 0; j < PRE_BS; ++j) preB[j] = ldg_stream(s0 + (PRE_BS + j) * SLOT);
+        // the rest of that unit is asked into L2 meanwhile (the SM may sit at the wait below for several microseconds
+        // while the previous kernel's last CTAs finish, with HBM partly idle)
+        // (asking for the CTA's second unit as well measured slower)
+        if (PRE_S > 2 * PRE_BS && lane == 0)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(s0 + 2 * PRE_BS * SLOT), "r"((u32)((PRE_S - 2 * PRE_BS) * SLOT)) : "memory");
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
