@@ -219,6 +219,29 @@ __device__ __noinline__ u64 poll_h(const u64* p, u32 epoch, Ctrl* ctrl, u32* ger
     }
 }
 
+// The last CTA's final pass: y = bf16(y_acc), y_acc = 0, in rounds of CB 16-byte loads per thread, all in flight together
+// (the CTA is alone on this, and a round costs a trip to L2).  A function of its own so that its registers do not weigh
+// on the kernel's main loops.
+template <int CB>
+__device__ __noinline__ void cast_y(float* y_acc, __nv_bfloat16* y, int n4, int tid) {
+    float4* ya = reinterpret_cast<float4*>(y_acc);
+    uint2* yo = reinterpret_cast<uint2*>(y);
+    for (int i0 = tid; i0 < n4; i0 += NTHREADS * CB) {
+        float4 v[CB];
+#pragma unroll
+        for (int u = 0; u < CB; ++u)
+            if (i0 + u * NTHREADS < n4) v[u] = __ldcg(ya + i0 + u * NTHREADS);
+#pragma unroll
+        for (int u = 0; u < CB; ++u) {
+            const int i = i0 + u * NTHREADS;
+            if (i < n4) {
+                yo[i] = make_uint2(pack2(split_bits(v[u].x, 0), split_bits(v[u].y, 0)), pack2(split_bits(v[u].z, 0), split_bits(v[u].w, 0)));
+                ya[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+    }
+}
+
 // Event timestamps for performance work: compiled in only with -DPOP_STREAM_TRACE (a build of its own);
 // slot `id` of the calling CTA gets the time at which its lane 0 passed the marker.
 #ifdef POP_STREAM_TRACE
@@ -925,29 +948,39 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                 } else {
                     // Candidate unit: approximate score and a bound of its error.  The warps' partial sums are
                     // added in fp64 (exact for all practical purposes); each partial sum comes from S tensor-core
-                    // steps whose error is bounded through the magnitudes seen (P.cstep).
+                    // steps whose error is bounded through the magnitudes seen (P.cstep).  From there on the value runs
+                    // in fp32 (this one warp is what the candidate units of a CTA wait for, and fp64 exponentials,
+                    // divisions and square roots made it the slowest stage at larger batches); what that costs in
+                    // accuracy is added to the bound, and every bound is rounded up.
                     const int c2 = 8 * hdr.y + ch;
                     const bool live = c2 < P.n_cand && nn < B;
                     double e2 = 0.0, d2 = 0.0;
                     if (live) {
-                        const double pmg = (double)P.wmax_cand[c2] * (double)ctrl->xmax[nn];
-                        const double pmu = (double)P.wmax_cand[P.n_cand + c2] * (double)ctrl->xmax[nn];
-                        double gs = 0.0, us = 0.0, dg = 0.0, du = 0.0;
+                        const float xm = ctrl->xmax[nn];
+                        const float pmg = P.wmax_cand[c2] * xm * 1.000001f;
+                        const float pmu = P.wmax_cand[P.n_cand + c2] * xm * 1.000001f;
+                        double gs = 0.0, us = 0.0;
+                        float dg = 0.f, du = 0.f;
 #pragma unroll
                         for (int ww = 0; ww < NCW; ++ww) {
                             gs += (double)pb[ww * PART_W + ch * BCAP + nn];
                             us += (double)pb[ww * PART_W + (ch + 8) * BCAP + nn];
-                            dg += fmax((double)pb[ww * PART_W + 16 * BCAP + ch * BCAP + nn], pmg);
-                            du += fmax((double)pb[ww * PART_W + 16 * BCAP + (ch + 8) * BCAP + nn], pmu);
+                            dg += fmaxf(pb[ww * PART_W + 16 * BCAP + ch * BCAP + nn], pmg);
+                            du += fmaxf(pb[ww * PART_W + 16 * BCAP + (ch + 8) * BCAP + nn], pmu);
                         }
-                        dg *= P.cstep;
-                        du *= P.cstep;
-                        const double hv = silu_f64(gs) * us;
-                        P.h[(size_t)nn * P.h_stride + P.n_ret_pad + c2] = h_word((float)hv, epoch);
-                        // |silu'| <= 1.1
-                        const double dh = 1.1 * dg * (fabs(us) + du) + fabs(silu_f64(gs)) * du + 1e-15 * fabs(hv);
-                        e2 = hv * hv;
-                        d2 = dh * dh;
+                        const float cs = __double2float_ru(P.cstep * 1.000002);      // (the fp32 sums above: 8 x 2^-24)
+                        dg *= cs;
+                        du *= cs;
+                        const float gf = (float)gs, uf = (float)us;
+                        const float sg = silu_f32(gf);
+                        const float hv = sg * uf;
+                        P.h[(size_t)nn * P.h_stride + P.n_ret_pad + c2] = h_word(hv, epoch);
+                        // |silu'| <= 1.1.  fp32 from the sums on: the rounding of gs moves silu by at most (1 + |gs|) / 2
+                        // last places, expf, the addition and the division by 3 more, in all below 4e-6 of the value
+                        // for gs > -30; below -30 the value itself is under 3e-12 |us|.
+                        const float dh = (1.1f * dg * (fabsf(uf) + du) + fabsf(sg) * du + 4e-6f * fabsf(hv) + 1e-11f * fabsf(uf)) * 1.000002f + 1e-37f;
+                        e2 = (double)hv * (double)hv;
+                        d2 = (double)dh * (double)dh;
                     }
                     // sum over the batch columns of the channel (BCAP consecutive lanes)
 #pragma unroll
@@ -956,11 +989,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
                         d2 += __shfl_xor_sync(0xffffffffu, d2, off);
                     }
                     if (nn == 0 && c2 < P.n_cand) {
+                        // square roots in fp32 where the operand is an ordinary fp32 number (relative error 1e-7)
+                        auto root = [](double v) -> double {
+                            return (v > 1e-30 && v < 1e30) ? (double)sqrtf((float)v) : sqrt(v);
+                        };
                         const double nc = P.norm_cand[c2];
-                        const double key = nc * sqrt(e2);
+                        const double key = nc * root(e2);
                         const float kf = (float)key;
                         // bound of |fp32 key - exact score|, rounded up
-                        const float mf = __double2float_ru(nc * sqrt(d2) * (1.0 + 1e-9) + key * 1.3e-7);
+                        const float mf = __double2float_ru(nc * root(d2) * (1.0 + 1e-6) + key * 4e-7);
                         P.km[c2] = make_uint2(__float_as_uint(kf), __float_as_uint(mf));
                     }
                 }
@@ -1328,14 +1365,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
             P.sync[SYNC_RF_DONE] = 0;
             P.sync[SYNC_EPOCH] = ctrl->epoch;
         }
-        float4* ya = reinterpret_cast<float4*>(P.y_acc);
-        uint2* yo = reinterpret_cast<uint2*>(P.y);
-#pragma unroll 4
-        for (int i = tid; i < (B * d) >> 2; i += NTHREADS) {
-            const float4 v = __ldcg(ya + i);
-            yo[i] = make_uint2(pack2(split_bits(v.x, 0), split_bits(v.y, 0)), pack2(split_bits(v.z, 0), split_bits(v.w, 0)));
-            ya[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+        cast_y<8 * NBLK>(P.y_acc, P.y, (B * d) >> 2, tid);
         if (warp == 0) POP_TRACE(18);
     }
 }
