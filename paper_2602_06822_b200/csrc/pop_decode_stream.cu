@@ -899,14 +899,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
         // the approximate score keys with their error bounds) and counts the candidate units done.
         // The consumer warps never wait for it.
         const u32 epoch = ld_acquire_gpu(P.sync + SYNC_EPOCH) + 1u;
-        // max |x[b][:]| for the error bounds of the candidate scores
+        // max |x[b][:]| for the error bounds of the candidate scores.  All loads of a row are in flight together (up to 20
+        // vectors per lane at d = 5120): one trip to memory per batch row (a loop of four loads at a time made this warp
+        // start on the first candidate unit 19 us late at batch 8).
         for (int bb = 0; bb < B; ++bb) {
-            float mx = 0.f;
             const uint4* xv = reinterpret_cast<const uint4*>(P.x + (size_t)bb * d);
-#pragma unroll 4
-            for (int v = lane; v < (d >> 3); v += 32) {
+            constexpr int XV = 4 * GS;                       // d / 8 / 32 vectors per lane (d = 1024 GS)
+            uint4 xr[XV];
+#pragma unroll
+            for (int v = 0; v < XV; ++v) xr[v] = __ldg(xv + lane + 32 * v);
+            float mx = 0.f;
+#pragma unroll
+            for (int v = 0; v < XV; ++v) {
                 float f[8];
-                Elem<__nv_bfloat16>::unpack(__ldg(xv + v), f);
+                Elem<__nv_bfloat16>::unpack(xr[v], f);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) mx = fmaxf(mx, fabsf(f[e]));
             }
