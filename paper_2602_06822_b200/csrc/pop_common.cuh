@@ -111,7 +111,7 @@ PopConfig pop_config_snapshot();
 
 // sync[] word assignment (contended counters sit on separate 128-byte lines)
 enum { SYNC_BARRIER = 0, SYNC_TICKET = 1, SYNC_ERROR = 2, SYNC_WORK = 3,
-       SYNC_EPOCH = 32, SYNC_CAND_DONE = 96,
+       SYNC_EPOCH = 32, SYNC_CAST_DONE = 64 /* CTAs done with their part of the final cast */, SYNC_CAND_DONE = 96,
        SYNC_Q0 = 128 /* + 32 q, q = 0..3 */, SYNC_QC0 = 256 /* + 32 q */, SYNC_RF_DONE = 384,
        SYNC_WORDS = 416 };
 

@@ -219,14 +219,14 @@ __device__ __noinline__ u64 poll_h(const u64* p, u32 epoch, Ctrl* ctrl, u32* ger
     }
 }
 
-// The last CTA's final pass: y = bf16(y_acc), y_acc = 0, in rounds of CB 16-byte loads per thread, all in flight together
+// The final pass of a CTA that finishes last: y = bf16(y_acc), y_acc = 0 over its part of the accumulator, in rounds of CB 16-byte loads per thread, all in flight together
 // (the CTA is alone on this, and a round costs a trip to L2).  A function of its own so that its registers do not weigh
 // on the kernel's main loops.
 template <int CB>
-__device__ __noinline__ void cast_y(float* y_acc, __nv_bfloat16* y, int n4, int tid) {
+__device__ __noinline__ void cast_y(float* y_acc, __nv_bfloat16* y, int lo4, int n4, int tid) {      // 16-byte groups [lo4, n4)
     float4* ya = reinterpret_cast<float4*>(y_acc);
     uint2* yo = reinterpret_cast<uint2*>(y);
-    for (int i0 = tid; i0 < n4; i0 += NTHREADS * CB) {
+    for (int i0 = lo4 + tid; i0 < n4; i0 += NTHREADS * CB) {
         float4 v[CB];
 #pragma unroll
         for (int u = 0; u < CB; ++u)
@@ -1353,25 +1353,50 @@ __global__ void __launch_bounds__(NTHREADS, 1) pop_decode_stream_kernel(const St
     // ========================================================================= finish
     __syncthreads();
     if (warp == 0) POP_TRACE(15);
+    // The CTAs that finish last cast the accumulator: one of them at small batches; at large ones (NBLK = 2: up to
+    // 8 d values, more than one SM moves in a microsecond) the last CAST_K share it, each waiting until every CTA has
+    // added its partial sums (they are the last to arrive, so the wait is short; it is bounded like every other).
+    constexpr int CAST_K_MAX = NBLK == 2 ? 8 : 1;
+    const int cast_k = CAST_K_MAX < G ? CAST_K_MAX : G;
     if (tid == 0) {
         const u32 ticket = atomicAdd(P.sync + SYNC_TICKET, 1u);
         __threadfence();
-        ctrl->last = (ticket == (u32)G - 1u) ? 1 : 0;
+        ctrl->last = (int)ticket - (G - cast_k) + 1;          // > 0: this CTA casts slice last - 1
     }
     __syncthreads();
-    if (ctrl->last) {
-        // every CTA has added its partial sums and is past its last use of the counters: re-arm them, advance the
-        // epoch (plain stores: the next launch on the stream starts only after this grid has completed), cast the
-        // accumulator and clear it
-        if (tid == 0) {
+    if (ctrl->last > 0) {
+        const int slice = ctrl->last - 1;
+        if (cast_k > 1) {
+            if (tid == 0) {
+                PopWaitClock sp;
+                while (ld_acquire_gpu(P.sync + SYNC_TICKET) < (u32)G) {
+                    if (sp.expired(P.wait_ns)) { atomicExch(gerr, (u32)ERR_THROTTLE); break; }
+                    __nanosleep(50);
+                }
+            }
+            __syncthreads();
+        }
+        // every CTA has added its partial sums: cast this CTA's part of the accumulator and clear it
+        const int n4 = (B * d) >> 2;
+        const int lo = (int)((long long)n4 * slice / cast_k), hi = (int)((long long)n4 * (slice + 1) / cast_k);
+        cast_y<8 * NBLK>(P.y_acc, P.y, lo, hi, tid);
+        bool rearm = cast_k == 1;
+        if (cast_k > 1) {
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) rearm = atomicAdd(P.sync + SYNC_CAST_DONE, 1u) == (u32)cast_k - 1u;
+        }
+        if (tid == 0 && rearm) {
+            // every CTA is past its last use of the counters: re-arm them and advance the epoch (plain stores: the
+            // next launch on the stream starts only after this grid has completed)
             P.sync[SYNC_TICKET] = 0;
+            P.sync[SYNC_CAST_DONE] = 0;
             P.sync[SYNC_CAND_DONE] = 0;
 #pragma unroll
             for (int q = 0; q < 4; ++q) { P.sync[SYNC_Q0 + 32 * q] = 0; P.sync[SYNC_QC0 + 32 * q] = 0; }
             P.sync[SYNC_RF_DONE] = 0;
             P.sync[SYNC_EPOCH] = ctrl->epoch;
         }
-        cast_y<8 * NBLK>(P.y_acc, P.y, (B * d) >> 2, tid);
         if (warp == 0) POP_TRACE(18);
     }
 }
