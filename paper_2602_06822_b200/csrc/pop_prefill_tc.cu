@@ -39,7 +39,7 @@ constexpr int TC_BN = 128;                 // tokens per unit
 constexpr int TC_BK = 64;                  // K slab of one pipeline stage: 64 bf16 = one 128-byte swizzle row
 constexpr int TC_STAGES = 4;
 constexpr int TC_CHUNK_SLABS = 1;          // accumulate-restart chunk = 64 hidden dimensions (4 MMAs)
-constexpr int TC_TRACK = 4;                // the running sums' magnitudes are sampled every TC_TRACK chunks
+constexpr int TC_TRACK = 8;                // the running sums' magnitudes are sampled every TC_TRACK chunks
 constexpr int TC_TILE_BYTES = TC_BM * TC_BK * 2;          // 16 KB
 constexpr int TC_STAGE_BYTES = 3 * TC_TILE_BYTES;         // Wg, Wu, X
 constexpr int TC_THREADS = 320;
@@ -82,10 +82,10 @@ __device__ __forceinline__ u32 mbar_try_wait(u32 bar, u32 parity) {
     u32 ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(2000u)      // the thread may stay suspended this long (ns) inside one try: fewer polls
         : "memory");
     return ok;
 }
@@ -309,24 +309,27 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
         const float eps = (float)(TC_CHUNK_SLABS * (TC_BK / 16)) * TC_KAPPA + (float)TC_TRACK * TC_ADD_ULP;
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
             const int ct = unit / P.n_tt, tt = unit - ct * P.n_tt;
-            float g[64], u[64];
+            // running sums in pairs: the chunk additions are packed fp32 additions (two round-to-nearest sums per
+            // instruction), which halves what the read-out costs the issue slots it shares with everything else
+            float2 g2[32], u2[32];
 #pragma unroll
-            for (int j = 0; j < 64; ++j) { g[j] = 0.f; u[j] = 0.f; }
+            for (int j = 0; j < 32; ++j) { g2[j] = make_float2(0.f, 0.f); u2[j] = make_float2(0.f, 0.f); }
             float track_g = 0.f, track_u = 0.f;           // sums of the sampled largest |running sum|
             for (int c = 0; c < n_chunks; ++c) {
                 ok = mbar_wait(bar_acc_full + 8 * buf, accph[buf], abortp, P.status, TC_ERR_EPILOGUE);
                 if (!ok) break;
                 tc_fence_after();
                 const u32 t_g = tmem_base + lane_base + (u32)buf * 256u + (u32)half * 64u, t_u = t_g + 128u;
+                // (two loads in flight at a time, the second under the additions of the first, measured no faster)
 #pragma unroll
                 for (int p = 0; p < 2; ++p) {
                     float v[32];
                     tmem_ld32(t_g + 32u * p, v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) g[32 * p + j] += v[j];
+                    for (int j = 0; j < 16; ++j) g2[16 * p + j] = __fadd2_rn(g2[16 * p + j], make_float2(v[2 * j], v[2 * j + 1]));
                     tmem_ld32(t_u + 32u * p, v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) u[32 * p + j] += v[j];
+                    for (int j = 0; j < 16; ++j) u2[16 * p + j] = __fadd2_rn(u2[16 * p + j], make_float2(v[2 * j], v[2 * j + 1]));
                 }
                 tc_fence_before();
                 __syncwarp();
@@ -336,7 +339,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
                 if ((c % TC_TRACK) == TC_TRACK - 1 || c == n_chunks - 1) {
                     float mg = 0.f, mu = 0.f;
 #pragma unroll
-                    for (int j = 0; j < 64; ++j) { mg = fmaxf(mg, fabsf(g[j])); mu = fmaxf(mu, fabsf(u[j])); }
+                    for (int j = 0; j < 32; ++j) {
+                        mg = fmaxf(mg, fmaxf(fabsf(g2[j].x), fabsf(g2[j].y)));
+                        mu = fmaxf(mu, fmaxf(fabsf(u2[j].x), fabsf(u2[j].y)));
+                    }
                     track_g += mg;
                     track_u += mu;
                 }
@@ -348,7 +354,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
             if (P.dump_g) {
                 const size_t o = (size_t)ch * (P.n_tt * TC_BN) + tt * TC_BN + half * 64;
 #pragma unroll
-                for (int j = 0; j < 64; ++j) { P.dump_g[o + j] = g[j]; P.dump_u[o + j] = u[j]; }
+                for (int j = 0; j < 64; ++j) { P.dump_g[o + j] = (j & 1) ? g2[j >> 1].y : g2[j >> 1].x; P.dump_u[o + j] = (j & 1) ? u2[j >> 1].y : u2[j >> 1].x; }
             }
 #endif
             const float cg = eps * P.gnorm[ch], cu = eps * P.unorm[ch];
@@ -364,7 +370,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) prefill_tc_kernel(const __grid_
             for (int j = 0; j < 64; ++j) {
                 const float at = __ldg(xn + j);
                 const float dg = at * cg + ag, du = at * cu + au;       // |g - exact|, |u - exact| at most these
-                const float gj = g[j], uj = u[j];
+                const float gj = (j & 1) ? g2[j >> 1].y : g2[j >> 1].x, uj = (j & 1) ? u2[j >> 1].y : u2[j >> 1].x;
                 const float e = __expf(-fmaxf(gj, -80.f));
                 const float s = gj * __fdividef(1.f, 1.f + e);          // silu(g)
                 const float h = s * uj;
