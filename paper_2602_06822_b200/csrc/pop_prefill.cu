@@ -735,8 +735,8 @@ __device__ __forceinline__ void rwd_emit(const unsigned short* __restrict__ W, c
     }
 }
 
-__global__ void __launch_bounds__(256) repack_wd_tiled_kernel(const __nv_bfloat16* __restrict__ Wd, int d, int N, int n_ret,
-                                                              int n_cg, int n_cand, const int32_t* __restrict__ idx_ret,
+__global__ void __launch_bounds__(256, 5) repack_wd_tiled_kernel(const __nv_bfloat16* __restrict__ Wd, int d, int N, int n_ret,
+                                                              int n_cg, int n_cand, int span_cap, const int32_t* __restrict__ idx_ret,
                                                               const int32_t* __restrict__ idx_cand, uint4* __restrict__ WdTt,
                                                               __nv_bfloat16* __restrict__ WdTc) {
     extern __shared__ __align__(16) unsigned short rwd_tile[];     // [RWD_ROWS][pitch]
@@ -754,7 +754,7 @@ __global__ void __launch_bounds__(256) repack_wd_tiled_kernel(const __nv_bfloat1
     const int c_hi = sg == n_sg - 1 ? N : __ldg(idx_ret + RWD_SLOTS * (sg + 1));
     const int c_lo8 = c_lo & ~7;
     const int nvec = (c_hi - c_lo8 + 7) >> 3;                       // 16-byte vectors per staged row (N is a multiple of 8)
-    const bool staged = nvec * 8 <= RWD_SPAN_MAX + 8;
+    const bool staged = nvec * 8 <= span_cap + 8;      // the launch sized the staging buffer for spans of span_cap channels
     const int pitch = 8 * rwd_pitch_vec(nvec);
     __syncthreads();
     if (staged) {
@@ -816,16 +816,22 @@ int pop_launch_repack_tiled(const pop_partition* p, const void* Wg, const void* 
     }
     const bool merged = repack_wd_tiled_applies(p);
     if (merged) {
-        const size_t smem = sizeof(unsigned short) * RWD_ROWS * 8 * rwd_pitch_vec(RWD_SPAN_MAX / 8 + 1);
+        // The staging buffer is sized for spans a quarter wider than the average one (128 N / n_ret channels), at most
+        // RWD_SPAN_MAX: a smaller buffer lets more blocks share an SM, and the kernel is bound by latency.
+        long long cap = ((long long)RWD_SLOTS * p->N * 5 / 4) / p->n_ret + 16;
+        int span_cap = (int)((cap + 7) / 8 * 8);
+        if (span_cap > RWD_SPAN_MAX) span_cap = RWD_SPAN_MAX;
+        const size_t smem = sizeof(unsigned short) * RWD_ROWS * 8 * rwd_pitch_vec(span_cap / 8 + 1);
         static thread_local int cfg_dev = -1;
         int dev = 0;
         POP_CUDA(cudaGetDevice(&dev));
         if (cfg_dev != dev) {
-            POP_CUDA(cudaFuncSetAttribute(repack_wd_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            const size_t smem_max = sizeof(unsigned short) * RWD_ROWS * 8 * rwd_pitch_vec(RWD_SPAN_MAX / 8 + 1);
+            POP_CUDA(cudaFuncSetAttribute(repack_wd_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max));
             cfg_dev = dev;
         }
         dim3 grd((p->n_ret + RWD_SLOTS - 1) / RWD_SLOTS, p->d / RWD_ROWS);
-        repack_wd_tiled_kernel<<<grd, 256, smem, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_ret, p->n_cg, p->n_cand,
+        repack_wd_tiled_kernel<<<grd, 256, smem, st>>>((const __nv_bfloat16*)Wd, p->d, p->N, p->n_ret, p->n_cg, p->n_cand, span_cap,
                                                        p->idx_ret, p->idx_cand, (uint4*)WdTt, (__nv_bfloat16*)WdTc);
         POP_LAUNCHED();
     } else if (p->n_rt > 0) {
