@@ -403,11 +403,16 @@ __device__ __noinline__ bool selection_main(const StreamParams& P, CtrlT<KPL>* c
             }
             for (int i = lane; i < 256; i += 32) hist[i] = 0;
             __syncwarp();
-#pragma unroll 4
-            for (int j = 0; j < rows; ++j) {
-                const u32 key = kr[32 * j];
-                if (lane + 32 * j < n && (key & mask) == prefix)
-                    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(hist_u + 4u * ((key >> shift) & 255u)), "r"(1u) : "memory");
+#pragma unroll 1
+            for (int j8 = 0; j8 < rows; j8 += 12) {
+                // twelve keys at a time: their loads from shared memory are issued together
+                u32 key[12];
+#pragma unroll
+                for (int t = 0; t < 12; ++t) key[t] = kr[32 * (j8 + t < KPL ? j8 + t : 0)];
+#pragma unroll
+                for (int t = 0; t < 12; ++t)
+                    if (j8 + t < rows && lane + 32 * (j8 + t) < n && (key[t] & mask) == prefix)
+                        asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(hist_u + 4u * ((key[t] >> shift) & 255u)), "r"(1u) : "memory");
             }
             __syncwarp();
             u32 c[8], tot = 0;
