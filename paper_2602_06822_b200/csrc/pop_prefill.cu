@@ -438,8 +438,8 @@ __global__ void __launch_bounds__(128) rank_list_kernel(const u64* __restrict__ 
 
 static int launch_ranks(const double* scores, int N, int32_t* rank, int sm_count, const int* run_if_gt, int threshold, cudaStream_t st) {
     const int bx = (N + 2 * RANK_NT - 1) / (2 * RANK_NT);
-    int by = (4 * sm_count + bx - 1) / bx;                                   // about four blocks per SM in all
-    const int max_by = (N + RANK_TILE - 1) / RANK_TILE;
+    int by = (8 * sm_count + bx - 1) / bx;                                   // about eight blocks per SM in all (the kernel is bound by latency: four took 39 us at N = 11008)
+    const int max_by = (N + 255) / 256;
     if (by > max_by) by = max_by;
     if (by < 1) by = 1;
     int j_chunk = (N + by - 1) / by;
@@ -499,8 +499,8 @@ int pop_launch_partition_after_rescore(const double* scores, int N, int n_ret, i
                                        const int32_t* list, const int* n_list, int max_list, int32_t* idx_ret,
                                        int32_t* idx_cand, int32_t* idx_pruned, cudaStream_t st) {
     // lists are short (blocks past the list's end return at once), so the channel axis is cut finely
-    int by = (N + 511) / 512;
-    if (by > 64) by = 64;
+    int by = (N + 255) / 256;
+    if (by > 128) by = 128;
     if (by < 1) by = 1;
     (void)sm_count;
     int j_chunk = (((N + by - 1) / by) + 255) & ~255;
