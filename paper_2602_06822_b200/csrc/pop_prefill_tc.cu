@@ -563,7 +563,12 @@ __global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* 
 // rescore_finish_kernel adds the groups in order.
 // Does nothing when the list is empty or longer than max_list (then the full fp64 pass runs instead).
 // ---------------------------------------------------------------------------------------------
-constexpr int RS_CH = 8, RS_WARPS = 4;
+constexpr int RS_CH = 8;
+// The four warps of a block share an item: each takes a quarter of the hidden size, and warp 0 adds the four partial
+// gate and up sums (in warp order) before the activation.  One warp per item was bound by the length of its dependent
+// fp64 MMA chains (84 us whatever the number of items); a quarter of the chain and four times the warps keep the fp64
+// tensor path busy.
+constexpr int RS_WARPS = 4;
 constexpr int RS_TOK_MIN = 16;             // token groups of the shortest items (part[] is sized for them)
 constexpr int RS_SHORT_LIST = 256;         // lists up to this length use 16-token items (more, shorter items)
 
@@ -583,9 +588,8 @@ template <int NA>
 __device__ __forceinline__ void rescore_item(const __nv_bfloat16* __restrict__ X, int L, int d,
                                              const __nv_bfloat16* __restrict__ Wg, const __nv_bfloat16* __restrict__ Wu,
                                              const int32_t* __restrict__ list, int n, int grp, int t0, int lane,
-                                             double& e0, double& e1) {
+                                             int kb_lo, int kb_hi, double (&g)[NA][2], double (&u)[NA][2]) {
     const int r = lane >> 2, c = lane & 3;
-    const int nkb = (d + 31) >> 5;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     const __nv_bfloat16* xr[NA];
 #pragma unroll
@@ -597,7 +601,6 @@ __device__ __forceinline__ void rescore_item(const __nv_bfloat16* __restrict__ X
     const int ch = li < n ? list[li] : -1;
     const __nv_bfloat16* wg = ch >= 0 ? Wg + (size_t)ch * d + 8 * c : nullptr;
     const __nv_bfloat16* wu = ch >= 0 ? Wu + (size_t)ch * d + 8 * c : nullptr;
-    double g[NA][2], u[NA][2];
 #pragma unroll
     for (int a = 0; a < NA; ++a) { g[a][0] = g[a][1] = u[a][0] = u[a][1] = 0.0; }
     uint4 vx[NA], vg, vu;
@@ -608,13 +611,13 @@ __device__ __forceinline__ void rescore_item(const __nv_bfloat16* __restrict__ X
         vg = (wg && in) ? __ldg(reinterpret_cast<const uint4*>(wg + (kb << 5))) : zero;
         vu = (wu && in) ? __ldg(reinterpret_cast<const uint4*>(wu + (kb << 5))) : zero;
     };
-    fetch(0);
-    for (int kb = 0; kb < nkb; ++kb) {
+    if (kb_lo < kb_hi) fetch(kb_lo);
+    for (int kb = kb_lo; kb < kb_hi; ++kb) {
         uint4 cx[NA];
 #pragma unroll
         for (int a = 0; a < NA; ++a) cx[a] = vx[a];
         const uint4 cg = vg, cu = vu;
-        if (kb + 1 < nkb) fetch(kb + 1);                // the next block's loads fly during this block's arithmetic
+        if (kb + 1 < kb_hi) fetch(kb + 1);                // the next block's loads fly during this block's arithmetic
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
             const double gb = bf16x8_elem(cg, s), ub = bf16x8_elem(cu, s);
@@ -626,8 +629,13 @@ __device__ __forceinline__ void rescore_item(const __nv_bfloat16* __restrict__ X
             }
         }
     }
-    // lane (r, c) holds token row r of each fragment at listed channels 2c, 2c + 1 of the group; tokens past L gave 0.
-    // Token sum: the fragments in the lane, then the 8 token rows (lanes r = 0..7 of the same c) by shuffles.
+}
+
+// The item's token sum from the complete gate and up sums: lane (r, c) holds token row r of each fragment at listed
+// channels 2c, 2c + 1 of the group (tokens past L gave 0); the fragments in the lane, then the 8 token rows (lanes
+// r = 0..7 of the same c) by shuffles.
+template <int NA>
+__device__ __forceinline__ void rescore_item_energy(const double (&g)[NA][2], const double (&u)[NA][2], double& e0, double& e1) {
     e0 = 0.0; e1 = 0.0;
 #pragma unroll
     for (int a = 0; a < NA; ++a) {
@@ -639,6 +647,42 @@ __device__ __forceinline__ void rescore_item(const __nv_bfloat16* __restrict__ X
     for (int off = 4; off < 32; off <<= 1) {
         e0 += __shfl_xor_sync(0xffffffffu, e0, off);
         e1 += __shfl_xor_sync(0xffffffffu, e1, off);
+    }
+}
+
+// One item by the block's RS_WARPS warps: partial sums over a share of the hidden size each, exchanged through shared
+// memory and added by warp 0 in warp order.
+template <int NA>
+__device__ __forceinline__ void rescore_block_item(const __nv_bfloat16* __restrict__ X, int L, int d,
+                                                   const __nv_bfloat16* __restrict__ Wg, const __nv_bfloat16* __restrict__ Wu,
+                                                   const int32_t* __restrict__ list, int n, int grp, int t0, int warp, int lane,
+                                                   double* xch, double& e0, double& e1) {
+    const int nkb = (d + 31) >> 5, per = (nkb + RS_WARPS - 1) / RS_WARPS;
+    double g[NA][2], u[NA][2];
+    rescore_item<NA>(X, L, d, Wg, Wu, list, n, grp, t0, lane, min(nkb, warp * per), min(nkb, (warp + 1) * per), g, u);
+    __syncthreads();                                   // the exchange buffer is free (the item before has been read)
+    if (warp > 0) {
+#pragma unroll
+        for (int a = 0; a < NA; ++a)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                xch[(((warp - 1) * NA + a) * 4 + h) * 32 + lane] = g[a][h];
+                xch[(((warp - 1) * NA + a) * 4 + 2 + h) * 32 + lane] = u[a][h];
+            }
+    }
+    __syncthreads();
+    e0 = 0.0; e1 = 0.0;
+    if (warp == 0) {
+#pragma unroll
+        for (int w = 1; w < RS_WARPS; ++w)
+#pragma unroll
+            for (int a = 0; a < NA; ++a)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    g[a][h] += xch[(((w - 1) * NA + a) * 4 + h) * 32 + lane];
+                    u[a][h] += xch[(((w - 1) * NA + a) * 4 + 2 + h) * 32 + lane];
+                }
+        rescore_item_energy<NA>(g, u, e0, e1);
     }
 }
 
@@ -657,11 +701,14 @@ __global__ void __launch_bounds__(32 * RS_WARPS) rescore_list_kernel(const __nv_
     const bool short_items = n <= RS_SHORT_LIST;
     const int n_tg = short_items ? n_tb : (n_tb + 1) / 2;
     const int items = n_grp * n_tg;
-    for (int item = blockIdx.x * RS_WARPS + (threadIdx.x >> 5); item < items; item += gridDim.x * RS_WARPS) {
+    __shared__ double xch[(RS_WARPS - 1) * 4 * 4 * 32];           // partial sums of warps 1.. for up to 4 fragments
+    const int warp = threadIdx.x >> 5;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
         const int grp = item / n_tg, tg = item - grp * n_tg;
         double e0, e1;
-        if (short_items) rescore_item<2>(X, L, d, Wg, Wu, list, n, grp, tg * 16, lane, e0, e1);
-        else rescore_item<4>(X, L, d, Wg, Wu, list, n, grp, tg * 32, lane, e0, e1);
+        if (short_items) rescore_block_item<2>(X, L, d, Wg, Wu, list, n, grp, tg * 16, warp, lane, xch, e0, e1);
+        else rescore_block_item<4>(X, L, d, Wg, Wu, list, n, grp, tg * 32, warp, lane, xch, e0, e1);
+        if (warp != 0) continue;
         if (r == 0) {
             const int l0 = grp * RS_CH + 2 * c;
             const int slot = short_items ? tg : 2 * tg;
@@ -1018,7 +1065,7 @@ int pop_launch_prefill_rescore(const void* X, int L, int d, const void* Wg, cons
     if (rc0 != POP_OK) return rc0;
     select_uncertain_kernel<<<1, SEL_NT, 0, st>>>(scores, bounds, s.rank, N, n_ret, n_cand, n_third, s.m_max, s.list, s.n_list);
     POP_LAUNCHED();
-    rescore_list_kernel<<<sm_count * 4, 32 * RS_WARPS, 0, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg,
+    rescore_list_kernel<<<sm_count * 8, 32 * RS_WARPS, 0, st>>>((const __nv_bfloat16*)X, L, d, (const __nv_bfloat16*)Wg,
                                                         (const __nv_bfloat16*)Wu, s.list, s.n_list, plan.max_list,
                                                         plan.n_tb, s.part);
     POP_LAUNCHED();
