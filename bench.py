@@ -412,6 +412,22 @@ def run_pop(args):
     def reduce_max(v):
         return max_over_ranks(v, world, dev)
 
+    # partial probing (Sec. 3.4): the same prefill from every fourth prompt token, outside the timed steps
+    probe_ms = None
+    if not args.no_variants:
+        torch = __import__("torch")
+        for rep in range(3):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            ev[0].record(stream)
+            pp = [WT[l].prefill_partition_probe(X, ratios, 4) for l in range(layers)]
+            ev[1].record(stream)
+            torch.cuda.synchronize()
+            for q in pp:
+                q.check()
+                q.destroy()
+            probe_ms = ev[0].elapsed_time(ev[1]) / layers
+        probe_ms = reduce_max(probe_ms)
+
     peaks = {}
     pk_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(pk_path):
@@ -536,6 +552,8 @@ def run_pop(args):
             "prefill_note": "pop_prefill_partition_prepared: the weight statistics (pop_weights_prepare) are computed once "
                             "per layer before the timed region; scoring on the tensor cores (tcgen05), exact re-scoring "
                             "of the channels near the rank boundaries, ranking, repack",
+            "prefill_probe": None if probe_ms is None else {"token_stride": 4, "ms_per_layer": probe_ms,
+                                                            "note": "pop_prefill_partition_probe: statistics from every 4th prompt token"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "layer-steps/s",
                     "h2d_bytes_per_step": int(X_host.numel() * es + tokens * B * d * es),

@@ -148,6 +148,18 @@ int pop_weights_prepare(const void* Wg, const void* Wu, const void* Wd, int N, i
                         void* cuda_stream, pop_weights_t** out);
 int pop_prefill_partition_prepared(const void* X, int L, const pop_weights_t* w, pop_ratios_t ratios,
                                    void* cuda_stream, pop_partition_t** out);
+
+/*
+ * Partial probing (Sec. 3.4 names "partial probing prompt activations" as the source of the prefill statistics
+ * without defining the subset; here: every token_stride-th prompt token, rows 0, token_stride, 2 token_stride, ...
+ * of X).  pop_prefill_partition_probe(X, L, s, w, ...) gives exactly the partition that
+ * pop_prefill_partition_prepared gives for those ceil(L / s) rows alone (s = 1: the whole prompt), at a cost that
+ * falls with s: the rows are gathered on the device into a temporary and scored from there.  X [L, d] device,
+ * row-major, 16-byte aligned; token_stride >= 1 (POP_ERR_INVALID_ARG otherwise).  Everything else as
+ * pop_prefill_partition_prepared.
+ */
+int pop_prefill_partition_probe(const void* X, int L, int token_stride, const pop_weights_t* w, pop_ratios_t ratios,
+                                void* cuda_stream, pop_partition_t** out);
 int pop_weights_destroy(pop_weights_t* w);
 
 /*

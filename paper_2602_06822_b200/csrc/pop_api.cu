@@ -366,7 +366,7 @@ extern "C" int pop_weights_destroy(pop_weights_t* w) {
 // are computed into this call's temporaries.
 static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, const void* Wu, const void* Wd, int N,
                                   pop_dtype_t dtype, pop_ratios_t ratios, const pop_weights* prepared, cudaStream_t st,
-                                  pop_partition_t** out, int k_out = -1, void* Y = nullptr) {
+                                  pop_partition_t** out, int k_out = -1, void* Y = nullptr, int token_stride = 1) {
     int n_ret, n_cand, n_pruned;
     int rc = pop_region_sizes(N, ratios, &n_ret, &n_cand, &n_pruned, nullptr);
     if (rc != POP_OK) return rc;
@@ -381,11 +381,15 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
 
     // temporaries (one stream-ordered allocation, freed in stream order): column norms, activation energies and,
     // for the tensor-core pass, its partial sums, bounds and the re-scoring list
+    // partial probing: the statistics come from every token_stride-th prompt token, gathered into a temporary
+    const int L_all = L;
+    if (token_stride > 1) L = (L + token_stride - 1) / token_stride;
     const bool tc = pop_prefill_tc_supported(d, dtype);
     const bool gemm = pop_prefill_s2_gemm_supported(d);
     PrefillTcPlan tp;
     pop_prefill_tc_plan(L, d, N, &tp);
     SlabPlan tmp;
+    const size_t t_probe = tmp.take(token_stride > 1 ? (size_t)L * d * p->es : 0);
     const size_t t_norm = tmp.take(prepared ? 0 : sizeof(double) * (size_t)N);
     const size_t t_s2 = tmp.take(tc ? 0 : sizeof(double) * (size_t)N);
     const size_t t_s2part = tmp.take(gemm ? sizeof(double) * (size_t)N * (size_t)pop_prefill_s2_gemm_splits(L) : 0);
@@ -409,12 +413,16 @@ static int prefill_partition_impl(const void* X, int L, int d, const void* Wg, c
         partition_free_now(p, st);
         return POP_ERR_ALLOC;
     }
+    if (token_stride > 1) {
+        rc = pop_launch_gather_rows(X, L_all, (size_t)d * p->es, token_stride, tb + t_probe, st);
+        X = tb + t_probe;
+    }
     WeightStats ws;
-    if (prepared) {
+    if (rc == POP_OK && prepared) {
         ws.norm = prepared->norm; ws.gnorm = prepared->gnorm; ws.unorm = prepared->unorm;
         ws.map_g = prepared->have_maps ? prepared->map_g : nullptr;
         ws.map_u = prepared->have_maps ? prepared->map_u : nullptr;
-    } else {
+    } else if (rc == POP_OK) {
         double* norm = (double*)(tb + t_norm);
         float *gn = (float*)(tb + t_gn), *un = (float*)(tb + t_un);
         rc = launch_weight_stats(Wg, Wu, Wd, N, d, dtype, norm, gn, un, tp.n_pad, st);
@@ -488,6 +496,18 @@ extern "C" int pop_prefill_partition_prepared(const void* X, int L, const pop_we
     POP_CUDA(cudaGetDevice(&dev));
     if (dev != w->device) return POP_ERR_INVALID_ARG;
     return prefill_partition_impl(X, L, w->d, w->Wg, w->Wu, w->Wd, w->N, w->dtype, ratios, w, (cudaStream_t)cuda_stream, out);
+}
+
+extern "C" int pop_prefill_partition_probe(const void* X, int L, int token_stride, const pop_weights_t* w, pop_ratios_t ratios,
+                                           void* cuda_stream, pop_partition_t** out) {
+    if (!out) return POP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!X || !w || L <= 0 || token_stride < 1 || !aligned16(X)) return POP_ERR_INVALID_ARG;
+    int dev = -1;
+    POP_CUDA(cudaGetDevice(&dev));
+    if (dev != w->device) return POP_ERR_INVALID_ARG;
+    return prefill_partition_impl(X, L, w->d, w->Wg, w->Wu, w->Wd, w->N, w->dtype, ratios, w, (cudaStream_t)cuda_stream, out,
+                                  -1, nullptr, token_stride);
 }
 
 extern "C" int pop_partition_from_indices(const void* Wg, const void* Wu, const void* Wd, int N, int d,

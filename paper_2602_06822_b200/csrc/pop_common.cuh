@@ -143,6 +143,7 @@ void pop_count_launch(int n);
 // ---------------------------------------------------------------------------------------------
 // pop_prefill.cu
 int pop_launch_colnorm(const void* Wd, int d, int N, pop_dtype_t dt, double* norm /*[N]*/, cudaStream_t st);
+int pop_launch_gather_rows(const void* X, int L, size_t row_bytes, int stride, void* Xp /*[ceil(L / stride)] rows*/, cudaStream_t st);
 int pop_launch_prefill_s2_exact(const void* X, int L, int d, const void* Wg, const void* Wu, int N,
                                 pop_dtype_t dt, const int32_t* chan_list /*NULL = all*/, int n_list,
                                 double* s2 /*[N], entries of listed channels are overwritten*/, cudaStream_t st);

@@ -33,6 +33,27 @@ __global__ void __launch_bounds__(1024) colnorm_kernel(const T* __restrict__ Wd,
     }
 }
 
+// Every stride-th row of X [L, row_bytes] (rows 0, stride, 2 stride, ...) into Xp, contiguous: the probe tokens of a
+// partial-probing prefill (Sec. 3.4).  16-byte vectors; row_bytes is a multiple of 16.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint4* __restrict__ X, int rows_out, int vec_per_row, int stride,
+                                                          uint4* __restrict__ Xp) {
+    const size_t total = (size_t)rows_out * vec_per_row;
+    for (size_t o = (size_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (size_t)gridDim.x * blockDim.x) {
+        const size_t r = o / vec_per_row, v = o - r * vec_per_row;
+        Xp[o] = __ldg(X + r * (size_t)stride * vec_per_row + v);
+    }
+}
+
+int pop_launch_gather_rows(const void* X, int L, size_t row_bytes, int stride, void* Xp, cudaStream_t st) {
+    const int rows_out = (L + stride - 1) / stride, vec = (int)(row_bytes / 16);
+    const size_t total = (size_t)rows_out * vec;
+    if (total == 0) return POP_OK;
+    const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+    gather_rows_kernel<<<blocks, 256, 0, st>>>((const uint4*)X, rows_out, vec, stride, (uint4*)Xp);
+    POP_LAUNCHED();
+    return POP_OK;
+}
+
 int pop_launch_colnorm(const void* Wd, int d, int N, pop_dtype_t dt, double* norm, cudaStream_t st) {
     dim3 blk(32, 32), grd((N + 31) / 32);
     if (dt == POP_F32) colnorm_kernel<float><<<grd, blk, 0, st>>>((const float*)Wd, d, N, norm);

@@ -64,6 +64,7 @@ SIGNATURES = {
                                         C.POINTER(_P)]),
     "pop_weights_prepare": (C.c_int, [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P, C.POINTER(_P)]),
     "pop_prefill_partition_prepared": (C.c_int, [_P, C.c_int, _P, Ratios, _P, C.POINTER(_P)]),
+    "pop_prefill_partition_probe": (C.c_int, [_P, C.c_int, C.c_int, _P, Ratios, _P, C.POINTER(_P)]),
     "pop_weights_destroy": (C.c_int, [_P]),
     "pop_prefill_partition_with_output": (C.c_int, [_P, C.c_int, _P, Ratios, C.c_int, _P, _P, C.POINTER(_P)]),
     "pop_partition_from_indices": (C.c_int, [_P, _P, _P, C.c_int, C.c_int, C.c_int, _P, C.c_int, _P, C.c_int,
@@ -294,6 +295,17 @@ class Weights:
         out = C.c_void_p()
         _check(lib().pop_prefill_partition_prepared(X.data_ptr(), X.shape[0], self._h, Ratios(*ratios), _stream_ptr(stream),
                                                     C.byref(out)), "pop_prefill_partition_prepared")
+        return Partition(out.value, X.device)
+
+    def prefill_partition_probe(self, X, ratios, token_stride: int, stream=None) -> "Partition":
+        """pop_prefill_partition_probe: the partition from every token_stride-th row of X [L, d]."""
+        if not (X.is_cuda and X.is_contiguous()) or _dtype_code(X) != _dtype_code(self.tensors[0]):
+            raise ValueError("X must be a contiguous CUDA tensor of the weights' dtype")
+        if X.shape[1] != self.tensors[0].shape[1]:
+            raise ValueError("shape mismatch")
+        out = C.c_void_p()
+        _check(lib().pop_prefill_partition_probe(X.data_ptr(), X.shape[0], int(token_stride), self._h, Ratios(*ratios),
+                                                 _stream_ptr(stream), C.byref(out)), "pop_prefill_partition_probe")
         return Partition(out.value, X.device)
 
     def prefill_partition_with_output(self, X, ratios, k: int, Y=None, stream=None):

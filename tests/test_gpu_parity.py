@@ -489,6 +489,31 @@ def test_prepared_weights_give_the_same_partition(d, N, L, dtype):
     wts.destroy()
 
 
+@pytest.mark.parametrize("d,N,L,stride,dtype", [(512, 1500, 70, 3, wl.BF16), (2048, 904, 200, 4, wl.BF16), (264, 777, 33, 2, wl.F32),
+                                                  (4096, 11008, 512, 4, wl.BF16), (1024, 1112, 64, 1, wl.BF16), (1024, 1112, 5, 7, wl.BF16)])
+def test_partial_probing_scores_every_s_th_token(d, N, L, stride, dtype):
+    """pop_prefill_partition_probe (Sec. 3.4 "partial probing prompt activations", read as every s-th prompt token): the
+    regions are those the oracle finds on rows 0, s, 2 s, ... of the prompt, the scores agree with it as those of a
+    whole prompt do, and the partition is the one pop_prefill_partition_prepared gives for those rows alone, bit for bit."""
+    cfg = wl.FFNConfig("probe", d=d, N=N, dtype=dtype, prompt_tokens=L, decode_steps=1, ratios=wl.Ratios(0.5, 0.2, 0.3), seed=d + stride)
+    w = wl.make_ffn_workload(cfg)
+    Wh = weights_host(w)
+    Wg, Wu, Wd = weights_dev(w)
+    wts = pop.Weights(Wg, Wu, Wd)
+    X = pr.to_dev(w.X)
+    a = wts.prefill_partition_probe(X, cfg.ratios.astuple(), stride)
+    ref = po.prefill_partition(w.X.values[::stride], *Wh, cfg.ratios.astuple())
+    check_prefill_scores(a, ref, dtype)
+    pr.check_regions(a, ref)
+    b = wts.prefill_partition(X[::stride].contiguous(), cfg.ratios.astuple())
+    for ia, ib in zip(a.indices(), b.indices()):
+        assert np.array_equal(ia, ib)
+    assert np.array_equal(a.scores(), b.scores()) and np.array_equal(a.score_bounds(), b.score_bounds())
+    with pytest.raises(pop.PopError):
+        wts.prefill_partition_probe(X, cfg.ratios.astuple(), 0)
+    a.destroy(); b.destroy(); wts.destroy()
+
+
 # ------------------------------------------------------------------ the prompt's own output under the pruned structure
 @pytest.mark.parametrize("d,N,L,kfrac", [(512, 1504, 70, 0.5), (2048, 904, 40, 0.25), (320, 648, 200, 1.0), (1024, 1112, 130, 0.0)])
 def test_prefill_output_small(d, N, L, kfrac):
