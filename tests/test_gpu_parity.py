@@ -355,6 +355,59 @@ def run_moe_case(cfg, n_experts, steps):
         part.destroy()
 
 
+def test_moe_batched_decode_groups_tokens_per_expert():
+    """Batched MoE decoding: the tokens of one step are grouped by routed expert and every group is one decode
+    step of that expert's partition, with one mask per group (candidate energy summed over the group's tokens, as
+    for any batch).  Checked group by group against the oracle's batched decode step, and token by token against the
+    router-weighted sum of the oracle's group outputs."""
+    cfg = wl.FFNConfig("moe_batch", d=2048, N=600, dtype=wl.BF16, prompt_tokens=48, decode_steps=8,
+                       ratios=wl.Ratios(0.5, 0.2, 0.3), seed=23)
+    n_experts = 4
+    m = wl.make_moe_workload(cfg, n_experts=n_experts, top_k=2, steps=8)
+    dev = torch.device("cuda:0")
+    ratios = cfg.ratios.astuple()
+    ex_host = [tuple(np.asarray(a.values, dtype=np.float64) for a in (e.Wg, e.Wu, e.Wd)) for e in m.experts]
+    ref_parts = po.moe_prefill_partitions(m.X.values, ex_host, m.prompt_logits, ratios, 2)
+    Xd = pr.to_dev(m.X)
+    parts = []
+    for e in range(n_experts):
+        tok = torch.from_numpy(np.asarray(ref_parts[e]["tokens"])).to(dev)
+        Wg, Wu, Wd = (pr.to_dev(a) for a in (m.experts[e].Wg, m.experts[e].Wu, m.experts[e].Wd))
+        part = pop.prefill_partition(Xd[tok].contiguous(), Wg, Wu, Wd, ratios)
+        pr.check_regions(part, ref_parts[e])
+        parts.append(part)
+    k = parts[0].n_cand // 2
+    xs = pr.to_dev(m.xs)[:, 0, :].contiguous()                      # the step's 8 tokens
+    xs_host = m.xs.values[:, 0, :]
+    ids, wts = po.moe_route(m.decode_logits, 2)                      # [8, 2] expert ids and renormalised weights
+    y = torch.zeros(8, cfg.d, dtype=torch.float64, device=dev)
+    y_ref = np.zeros((8, cfg.d))
+    groups = 0
+    for e in range(n_experts):
+        tok = np.nonzero((ids == e).any(axis=1))[0]
+        if tok.size == 0:
+            continue
+        groups += 1
+        R, C, _ = parts[e].indices()
+        mask = torch.empty(parts[e].n_cand, dtype=torch.uint8, device=dev)
+        sel = torch.empty(k, dtype=torch.int32, device=dev)
+        ye = pop.decode_step(parts[e], xs[torch.from_numpy(tok).to(dev)].contiguous(), k, mask_out=mask, sel_out=sel)
+        torch.cuda.synchronize()
+        parts[e].check()
+        oe = po.decode_step(xs_host[tok], *ex_host[e], ref_parts[e]["R"], ref_parts[e]["C"], k)
+        pr.check_selection(sel.cpu().numpy(), mask.cpu().numpy(), C, oe, k)
+        assert pr.rel_err(pr.host_values(ye), oe["y"], pr.FLOOR[cfg.dtype]) <= pr.TOL[cfg.dtype]
+        for g, t in enumerate(tok):
+            wt = float(wts[t][ids[t] == e][0])
+            y[t] += wt * ye[g].double()
+            y_ref[t] += wt * oe["y"][g]
+    assert groups >= 2
+    for t in range(8):
+        assert pr.normwise_err(y[t].cpu().numpy(), y_ref[t]) <= 1e-2
+    for part in parts:
+        part.destroy()
+
+
 def test_moe_small():
     cfg = wl.FFNConfig("moe_small", d=2048, N=600, dtype=wl.BF16, prompt_tokens=48, decode_steps=3,
                        ratios=wl.Ratios(0.5, 0.2, 0.3), seed=11)
