@@ -187,6 +187,17 @@ def prefill_partition(X, Wg, Wu, Wd, ratios: Sequence[float]) -> Dict[str, np.nd
     return {"scores": I, "R": R, "C": C, "P": P}
 
 
+def prefill_partition_probe(X, Wg, Wu, Wd, ratios: Sequence[float], token_stride: int) -> Dict[str, np.ndarray]:
+    """Prefilling stage from "partial probing prompt activations" (Sec. 3.4, which does not define the subset): read as
+    every token_stride-th prompt token, rows 0, s, 2s, ... of X.  Eq. 3 over those tokens only; stride 1 is the
+    whole prompt."""
+    if token_stride < 1:
+        raise ValueError("token_stride must be at least 1")
+    out = prefill_partition(_f64(X)[::token_stride], Wg, Wu, Wd, ratios)
+    out["tokens"] = np.arange(0, np.asarray(X).shape[0], token_stride)
+    return out
+
+
 # ----------------------------------------------------------------------------- decode step
 def candidate_scores(H_C: np.ndarray, Wd, C: np.ndarray) -> np.ndarray:
     """I_i(t), i in C, from this step's activations H_C [B, n_C] (Eq. 3 with the

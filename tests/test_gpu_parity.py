@@ -555,7 +555,7 @@ def test_partial_probing_scores_every_s_th_token(d, N, L, stride, dtype):
     wts = pop.Weights(Wg, Wu, Wd)
     X = pr.to_dev(w.X)
     a = wts.prefill_partition_probe(X, cfg.ratios.astuple(), stride)
-    ref = po.prefill_partition(w.X.values[::stride], *Wh, cfg.ratios.astuple())
+    ref = po.prefill_partition_probe(w.X.values, *Wh, cfg.ratios.astuple(), stride)
     check_prefill_scores(a, ref, dtype)
     pr.check_regions(a, ref)
     b = wts.prefill_partition(X[::stride].contiguous(), cfg.ratios.astuple())

@@ -358,3 +358,28 @@ def test_pins_catch_planted_mistakes(monkeypatch, mutation):
         monkeypatch.setattr(po, "channel_importance", lambda Wc, s: np.asarray(s, np.float64))
     with pytest.raises(AssertionError):
         test_hand_worked_example()
+
+
+def test_partial_probing_is_the_statistic_over_the_probe_tokens():
+    """Reading of Sec. 3.4 "partial probing": every s-th token.  Stride 1 is the whole prompt; a stride of L leaves the
+    first token alone, for which Eq. 3 is |h_i(x_0)| * |Wd[:, i]| written out; a channel that is active only on skipped
+    tokens scores zero."""
+    rng = np.random.default_rng(5)
+    L, d, N = 9, 6, 12
+    X = rng.standard_normal((L, d)); Wg = rng.standard_normal((N, d)); Wu = rng.standard_normal((N, d)); Wd = rng.standard_normal((d, N))
+    ratios = (0.5, 0.25, 0.25)
+    full = po.prefill_partition(X, Wg, Wu, Wd, ratios)
+    one = po.prefill_partition_probe(X, Wg, Wu, Wd, ratios, 1)
+    assert np.array_equal(full["scores"], one["scores"]) and np.array_equal(one["tokens"], np.arange(L))
+    first = po.prefill_partition_probe(X, Wg, Wu, Wd, ratios, L)
+    g, u = Wg @ X[0], Wu @ X[0]
+    h = g / (1.0 + np.exp(-g)) * u
+    assert np.allclose(first["scores"], np.abs(h) * np.linalg.norm(Wd, axis=0), rtol=1e-12)
+    assert np.array_equal(first["tokens"], [0])
+    third = po.prefill_partition_probe(X, Wg, Wu, Wd, ratios, 3)
+    assert np.array_equal(third["tokens"], [0, 3, 6])
+    Xz = X.copy(); Xz[[0, 3, 6]] = 0.0                      # the probe tokens silent: every score is zero
+    assert np.all(po.prefill_partition_probe(Xz, Wg, Wu, Wd, ratios, 3)["scores"] == 0.0)
+    assert np.any(po.prefill_partition(Xz, Wg, Wu, Wd, ratios)["scores"] > 0.0)
+    with pytest.raises(ValueError):
+        po.prefill_partition_probe(X, Wg, Wu, Wd, ratios, 0)
