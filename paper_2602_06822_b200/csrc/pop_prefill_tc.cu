@@ -510,7 +510,7 @@ __global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* 
     if (tid < 3) { mw_bits[tid] = 0ull; tau_sm[tid] = 0.0; }
     __syncthreads();
     // tau = the streamed score of the channel at rank n - 1 (exactly one channel holds each rank)
-    for (int i = lo; i < hi; ++i) {
+    for (int i = tid; i < N; i += SEL_NT) {                  // (coalesced: which thread finds them does not matter)
         const int r = rank[i];
         if (b1 && r == n1 - 1) tau_sm[0] = scores[i];
         if (b2 && r == n2 - 1) tau_sm[1] = scores[i];
@@ -524,7 +524,7 @@ __global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* 
     // outside, by the same two counts.
     const double w = 2.0 * m * (1.0 + 1e-9);
     double mw1 = 0.0, mw2 = 0.0, mw3 = 0.0;
-    for (int i = lo; i < hi; ++i) {
+    for (int i = tid; i < N; i += SEL_NT) {
         const double a = scores[i], mi = bounds[i];
         if (b1 && fabs(a - tau1) <= w) mw1 = fmax(mw1, mi);
         if (b2 && fabs(a - tau2) <= w) mw2 = fmax(mw2, mi);
@@ -541,12 +541,27 @@ __global__ void __launch_bounds__(SEL_NT) select_uncertain_kernel(const double* 
         return (b1 && fabs(a - tau1) <= w && fabs(a - tau1) <= mi + mw1) || (b2 && fabs(a - tau2) <= w && fabs(a - tau2) <= mi + mw2) ||
                (b3 && fabs(a - tau3) <= w && fabs(a - tau3) <= mi + mw3);
     };
+    // the list ascends: every thread a contiguous chunk of channels, read once (the open ones as a bit mask when the
+    // chunk has at most 64 channels)
     int cnt = 0;
-    for (int i = lo; i < hi; ++i) cnt += open_at(scores[i], bounds[i]);
+    u64 open_bits = 0ull;
+    for (int i = lo; i < hi; ++i) {
+        const bool o = open_at(scores[i], bounds[i]);
+        cnt += o;
+        if (o && i - lo < 64) open_bits |= 1ull << (i - lo);
+    }
     int tot;
     int pos = group_excl_scan<SEL_NT>(cnt, sm, tid, 0, tot);
-    for (int i = lo; i < hi; ++i) {
-        if (open_at(scores[i], bounds[i])) list[pos++] = i;
+    if (per <= 64) {
+        while (open_bits) {
+            const int b = __ffsll((long long)open_bits) - 1;
+            list[pos++] = lo + b;
+            open_bits &= open_bits - 1ull;
+        }
+    } else {
+        for (int i = lo; i < hi; ++i) {
+            if (open_at(scores[i], bounds[i])) list[pos++] = i;
+        }
     }
     if (tid == 0) *n_list = tot;
 }
